@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the USV sparsified-attention hot path on B200.
+
+One "step" = one pass of the attention path of the workload over one synthetic batch:
+block pooling + scores -> top-k key-block selection -> block-sparse attention forward
+(and, for the merging workloads, token merge before and token unmerge after).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl usv|reference]
+
+Prints ONE JSON line (rank 0).  `value` is dense-equivalent TFLOP/s of the whole job
+(4*B*H*N^2*d per step and rank, summed over ranks, divided by the max-over-ranks step time)
+with inputs resident in HBM; `e2e` is the same metric through the public API with pinned HOST
+buffers (H2D of q,k,v and D2H of o inside the timed region).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import usv_inputs as ui  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_BF16_TFLOPS = 2250.0
+PAPER_CONTEXT = ("paper: 83.3x DiT-denoising / 22.7x end-to-end speedup vs dense Wan2.1-1.3B "
+                 "(sparsity 0.95, 3 steps vs 50) on 1x NVIDIA H20, precision unstated; "
+                 "no kernel-level number is published")
+
+# DRAM bytes per launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum)
+# from the ncu capture summarised under profiles/; None until a capture exists for a workload.
+ATTN_DRAM_TRAFFIC = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.2] or [l for (_, l) in self.lines[-3:]]
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for nme, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w": float(np.median(power)) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def flops(wl, N, k_per_head):
+    """(dense-equivalent, effective) attention FLOPs of one call at sequence length N."""
+    NB = (N + 63) // 64
+    n_pad = NB * 64
+    dense = 4.0 * wl.B * wl.H * float(n_pad) ** 2 * wl.d
+    eff = 4.0 * wl.B * sum(float(n_pad) * 64 * k * wl.d for k in k_per_head)
+    return dense, eff
+
+
+def build_inputs(wl, device):
+    """Device-resident inputs of one step.  Returns a dict."""
+    if wl.merge_part is None:
+        q, k, v = ui.make_qkv(wl, device=device, layout="bhnd")
+        return dict(q=q, k=k, v=v, N=wl.N)
+    z = ui.make_hidden(wl, device)                                   # [B,N,C]
+    w = ui.make_qkv_weight(wl, device)                               # [C,3C]
+    metric = (z @ w[:, wl.C:2 * wl.C]).reshape(wl.B, wl.N, wl.H, wl.d).contiguous()
+    return dict(z=z, w=w, metric=metric, N=wl.N_attn)
+
+
+def run_usv(args, wl, rank, world, device):
+    import paper_2512_05754_b200 as usv
+    peaks, peak_src = load_peaks()
+    inp = build_inputs(wl, device)
+    kph = wl.k_per_head()
+    N = inp["N"]
+    dense_f, eff_f = flops(wl, N, kph)
+    merging = wl.merge_part is not None
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    if merging:
+        # projection of the merged hidden states is harness work (outside the library); it is
+        # done once, untimed, so that the timed step holds only the library's kernels.
+        zm, plan = usv.token_merge(inp["z"], inp["metric"], wl.grid, wl.merge_part, wl.r)
+        qkv = (zm @ inp["w"]).reshape(wl.B, N, 3, wl.H, wl.d)
+        q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))   # [B,H,N,d] views
+        o = torch.empty((wl.B, N, wl.H, wl.d), dtype=torch.bfloat16, device=device).permute(0, 2, 1, 3)
+    else:
+        q, k, v = inp["q"], inp["k"], inp["v"]
+        o = torch.empty_like(q)
+
+    marks = []
+
+    def step(record=False):
+        e = [ev() for _ in range(6)] if record else None
+        if record: e[0].record()
+        if merging:
+            usv.token_merge(inp["z"], inp["metric"], wl.grid, wl.merge_part, wl.r)
+        if record: e[1].record()
+        s = usv.block_scores(q, k, N, N)
+        if record: e[2].record()
+        sel = usv.select_blocks(s, kph)
+        if record: e[3].record()
+        usv.sparse_attn_fwd(q, k, v, sel, kph, N=N, out=o)
+        if record: e[4].record()
+        if merging:
+            usv.token_unmerge(o.permute(0, 2, 1, 3).reshape(wl.B, N, wl.C), plan.pos)
+        if record:
+            e[5].record()
+            marks.append(e)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(device.index)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    t_wall0 = time.time()
+    e0, e1 = ev(), ev()
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step(record=True)
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    total_ms = e0.elapsed_time(e1)
+    seg = np.array([[m[i].elapsed_time(m[i + 1]) for i in range(5)] for m in marks])  # ms
+    seg_mean = seg.mean(0)
+    assert usv.workspace_status() == 0
+
+    # ---- end to end through the public API with pinned host buffers
+    hq, hk, hv = (t.contiguous().cpu().pin_memory() for t in (q, k, v))
+    ho = torch.empty(o.shape, dtype=o.dtype).pin_memory()
+    dq, dk, dv = (torch.empty_like(t, device=device) for t in (hq, hk, hv))
+    do = torch.empty_like(dq)
+
+    def e2e_step():
+        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+        s = usv.block_scores(dq, dk, N, N)
+        sel = usv.select_blocks(s, kph)
+        usv.sparse_attn_fwd(dq, dk, dv, sel, kph, N=N, out=do)
+        ho.copy_(do, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    f0, f1 = ev(), ev()
+    f0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    f1.record()
+    barrier()
+    e2e_ms = f0.elapsed_time(f1) / e2e_steps
+
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
+    total_ms, e2e_ms = times.tolist()
+    if rank != 0:
+        return None
+    ms_step = total_ms / args.steps
+    attn_ms = float(seg_mean[3])
+    peak = peaks["bf16_tflops"]
+    attn_eff_tflops = eff_f / (attn_ms * 1e-3) / 1e12
+    launches_per_step = 4 + (8 + 1 if merging else 0)
+    hbm = peaks["hbm_gbs"]
+    pool_bytes = 2 * (wl.B * wl.H * N * wl.d * 2) + 2 * (wl.B * wl.H * ((N + 63) // 64) * wl.d * 4)
+    result = {
+        "metric": "sparse_attn_dense_equiv_tflops",
+        "value": world * dense_f / (ms_step * 1e-3) / 1e12,
+        "unit": "TFLOP/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step,
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "d": wl.d, "N": N,
+                   "blocks": (N + 63) // 64, "k_per_head": sorted(set(kph)),
+                   "merge_r": wl.r, "per_gpu": "one layer instance per GPU (heads/batch shard, no collective)",
+                   "l2": "inputs larger than L2 (q,k,v,o = %.0f MB per step), no flush" % (4 * q.numel() * 2 / 1e6)},
+        "breakdown_ms": {"token_merge": float(seg_mean[0]), "block_scores": float(seg_mean[1]),
+                         "select_blocks": float(seg_mean[2]), "sparse_attn_fwd": attn_ms,
+                         "token_unmerge": float(seg_mean[4]),
+                         "sparse_attn_fwd_min": float(seg[:, 3].min())},
+        "effective_tflops": {"attn_kernel": attn_eff_tflops,
+                             "step": eff_f / (ms_step * 1e-3) / 1e12,
+                             "frac_of_measured_burst": attn_eff_tflops / peak,
+                             "frac_of_measured_sustained": attn_eff_tflops / peaks["bf16_tflops_sustained"],
+                             "frac_of_nominal_2250": attn_eff_tflops / NOMINAL_BF16_TFLOPS},
+        "hbm": {"block_scores_GBps": pool_bytes / (seg_mean[1] * 1e-3) / 1e9,
+                "block_scores_frac": pool_bytes / (seg_mean[1] * 1e-3) / 1e9 / hbm},
+        "roofline": {"bound": "tensor", "kernel": "sparse_attn_fwd",
+                     "achieved": attn_eff_tflops, "peak": peak, "unit": "TFLOP/s",
+                     "frac": attn_eff_tflops / peak, "peak_source": "%s (burst bf16)" % peak_src,
+                     "traffic": ATTN_DRAM_TRAFFIC.get(wl.name)},
+        "e2e": {"value": world * dense_f / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(3 * hq.numel() * 2), "d2h_bytes_per_step": int(ho.numel() * 2)},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks,
+        "context": PAPER_CONTEXT,
+    }
+    if merging:
+        mb = (wl.B * wl.N * wl.C * 2) + (wl.B * N * wl.C * 2)
+        result["hbm"]["token_unmerge_GBps"] = mb / (seg_mean[4] * 1e-3) / 1e9
+        result["hbm"]["token_unmerge_frac"] = result["hbm"]["token_unmerge_GBps"] / hbm
+    return result, dict(q=q, k=k, v=v, N=N, kph=kph)
+
+
+def oracle_sample_step(wl, q, k, v, N, kph, n_qb, seed):
+    """One oracle pass: pooling, scores, selection in full; attention on n_qb sampled query
+    blocks.  Returns (seconds pooled/selected, seconds attention sample, blocks total)."""
+    import oracle
+    t0 = time.time()
+    s = oracle.block_scores(oracle.block_pool(q, N), oracle.block_pool(k, N))
+    sel, _ = oracle.select_blocks(s, kph)
+    t1 = time.time()
+    NB = (N + 63) // 64
+    allqb = oracle.all_query_blocks(wl.B, wl.H, NB)
+    rng = np.random.default_rng(seed)
+    pick = allqb[np.sort(rng.choice(allqb.shape[0], size=min(n_qb, allqb.shape[0]), replace=False))]
+    oracle.sparse_attn(q, k, v, N, sel, kph, qb_list=pick)
+    t2 = time.time()
+    return t1 - t0, t2 - t1, allqb.shape[0], pick.shape[0]
+
+
+def cpu_baseline(wl, tensors, n_qb=384):
+    import oracle
+    q, k, v = (tensors[n].contiguous().cpu() for n in ("q", "k", "v"))
+    N, kph = tensors["N"], tensors["kph"]
+    t_sel, t_attn, total, picked = oracle_sample_step(wl, q, k, v, N, kph, n_qb, 0)
+    t_full = t_sel + t_attn * total / picked
+    dense_f, _ = flops(wl, N, kph)
+    return {"value": dense_f / t_full / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "seconds_full_step_extrapolated": t_full,
+            "sample": "pooling+scores+selection in full (%.2f s); attention on %d of %d query "
+                      "blocks (%.2f s), extrapolated linearly" % (t_sel, picked, total, t_attn)}
+
+
+def run_reference(args, wl):
+    """The fp64 oracle as it stands, on host cores, same metric; each step a bounded sample."""
+    import oracle
+    q, k, v = ui.make_qkv(wl, device="cpu", layout="bhnd") if wl.merge_part is None else (None,) * 3
+    if q is None:
+        z = ui.make_hidden(wl, "cpu")
+        w = ui.make_qkv_weight(wl, "cpu")
+        metric = (z.float() @ w[:, wl.C:2 * wl.C].float()).to(torch.bfloat16).reshape(wl.B, wl.N, wl.H, wl.d)
+        plan = oracle.merge_plan(metric, wl.grid, wl.merge_part, wl.r)
+        zm = torch.from_numpy(oracle.round_to_bf16(oracle.merge_apply(z, plan["dst_of"], plan["pos"], plan["Nm"]))
+                              .view(np.int16)).view(torch.bfloat16)
+        qkv = (zm.float() @ w.float()).to(torch.bfloat16).reshape(wl.B, wl.N_attn, 3, wl.H, wl.d)
+        q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3).contiguous() for i in range(3))
+    N, kph = wl.N_attn, wl.k_per_head()
+    dense_f, _ = flops(wl, N, kph)
+    n_qb = 96
+    est = []
+    for i in range(args.warmup + args.steps):
+        t_sel, t_attn, total, picked = oracle_sample_step(wl, q, k, v, N, kph, n_qb, i)
+        if i >= args.warmup:
+            est.append(t_sel + t_attn * total / picked)
+    t_full = float(np.mean(est))
+    val = dense_f / t_full / 1e12
+    sample = ("each step: pooling+scores+selection in full, attention on %d of %d query blocks, "
+              "extrapolated linearly to the full call" % (picked, total))
+    return {"impl": "reference", "metric": "sparse_attn_dense_equiv_tflops", "value": val,
+            "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": t_full * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "d": wl.d, "N": N},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.num_threads(),
+                             "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="wan1.3b_480p")
+    ap.add_argument("--impl", default="usv", choices=["usv", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "usv" else args.warmup
+    wl = ui.workload(args.workload)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args, wl)))
+        return 0
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the product and has no CPU fallback")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=device)
+    out = run_usv(args, wl, rank, world, device)
+    if rank == 0:
+        result, tensors = out
+        if not args.no_cpu_baseline:
+            result["cpu_baseline"] = cpu_baseline(wl, tensors)
+        print(json.dumps(result))
+    if world > 1:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

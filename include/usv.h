@@ -1,0 +1,150 @@
+/*
+ * usv.h -- C ABI of the USV sparsified-attention hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, as hand-written CUDA kernels, one sparsified self-attention block of
+ * a video diffusion transformer as the USV paper describes it (Fig. 2 right; Sec. 3.2-3.3):
+ *
+ *     token merge -> block pooling + scores -> top-k key-block selection
+ *                 -> block-sparse attention -> token unmerge
+ *
+ * Conventions that hold for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned.  Arguments
+ *     documented as HOST are ordinary host pointers read before the call returns.
+ *   - Nothing is allocated, nothing is freed, the stream is never synchronised: kernels are
+ *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream).
+ *     Scratch memory comes from the caller (`ws`, `ws_bytes`); the matching *_workspace()
+ *     function gives the size needed.  The workspace may be reused by a later call on the same
+ *     stream; concurrent calls on different streams need different workspaces.
+ *   - Every function returns a usv_status.  Arguments are validated on the host before anything
+ *     is launched; on a non-zero status nothing has been enqueued (USV_ERR_CUDA excepted, which
+ *     reports a failed launch).  usv_last_error() gives a human-readable reason for the calling
+ *     thread's last failure.
+ *   - bf16 = the upper 16 bits of an IEEE binary32 value, round-to-nearest-even on output.
+ *   - Attention blocks are runs of USV_BLOCK = 64 consecutive tokens in the caller's token
+ *     order.  A sequence of N tokens has NB = ceil(N/64) blocks; the last one may be partial.
+ *     Rows at or beyond N are never read and never written.
+ *   - 4-d views [B,H,N,d] are described by element strides (sb, sh, sn) with the d axis
+ *     contiguous; strides must be multiples of 8 elements (16 bytes).
+ */
+#ifndef USV_H_
+#define USV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define USV_BLOCK 64
+#define USV_MAX_HEADS 128
+
+typedef enum {
+    USV_OK = 0,
+    USV_ERR_INVALID_ARG = 1, /* null pointer, bad size, k or r out of range ... */
+    USV_ERR_UNSUPPORTED = 2, /* valid request outside what the kernels cover (d, alignment) */
+    USV_ERR_WORKSPACE = 3,   /* ws_bytes smaller than *_workspace() */
+    USV_ERR_CUDA = 4,        /* a CUDA runtime/driver call or a launch failed */
+    USV_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (see usv_workspace_status) */
+} usv_status;
+
+/* Element strides of a [B,H,N,d] view whose d axis is contiguous. */
+typedef struct {
+    int64_t sb, sh, sn;
+} usv_strides;
+
+const char* usv_status_string(int status);
+const char* usv_last_error(void);
+/* Compiled-in build tag, e.g. "usv-b200 sm_100a". */
+const char* usv_build_info(void);
+
+/* ------------------------------------------------------------------------------------------
+ * Coarse stage of "top-k cube selection" (Fig. 2 caption; the paper names the step and leaves
+ * the score open).  Reading implemented: per 64-token block the mean of the valid query rows
+ * and of the valid key rows (fp32), then
+ *     scores[b,h,I,J] = < mean_q[b,h,I,:], mean_k[b,h,J,:] > / sqrt(d)          (fp32).
+ *
+ * q: bf16 view [B,H,Nq,d], k: bf16 view [B,H,Nk,d]; d in {64,128}.
+ * scores: fp32 [B,H,NBq,NBk] contiguous (written).  ws: pooled means, see *_workspace().
+ */
+size_t usv_block_scores_workspace(int B, int H, int Nq, int Nk, int d);
+int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void* q, const usv_strides* sq,
+                     const void* k, const usv_strides* sk, float* scores, void* ws,
+                     size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Top-k key-block selection (Fig. 2 caption, "top-k cube selection").  For each (b,h,I) the
+ * k_per_head[h] key blocks with the largest score are kept; equal scores are resolved in favour
+ * of the lower block index.  The kept indices are written in ascending order; the remainder of
+ * the kmax-wide row is filled with -1.
+ *
+ * scores: fp32 [B,H,NBq,NBk].  k_per_head: HOST int32[H], each in [1,NBk].  kmax >= max k.
+ * sel: int32 [B,H,NBq,kmax] (written).  NBk <= 8192.
+ */
+int usv_select_blocks(int B, int H, int NBq, int NBk, const float* scores,
+                      const int32_t* k_per_head, int kmax, int32_t* sel, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Block-sparse attention forward (Sec. 3.2, Eq. 5 with a block-structured mask):
+ *     O_i = sum_j softmax_j( scale * <q_i,k_j> ) v_j ,  j over the valid keys of the key blocks
+ *     listed in sel[b,h,block(i),0..k_per_head[h]).
+ * bf16 operands on the tensor cores, fp32 online softmax and accumulation, bf16 output.
+ *
+ * q,k,v: bf16 views [B,H,N,d] (self-attention: one N); d in {64,128}.
+ * sel: int32 [B,H,NB,kmax], entries in [0,NB), -1 entries are skipped.
+ * k_per_head: HOST int32[H].  o: bf16 view [B,H,N,d] (written, rows < N only).
+ * o_f32: optional fp32 [B,H,N,d] contiguous copy of the un-rounded output (NULL to skip).
+ * lse: optional fp32 [B,H,N], natural-log of the softmax denominator (NULL to skip).
+ * scale: logit scale; 0 selects 1/sqrt(d).
+ * impl: 0 = default kernel, 1 = legacy mma.sync kernel (kept as an on-device cross-check).
+ */
+size_t usv_sparse_attn_workspace(int B, int H, int N, int d, int kmax);
+int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,
+                        const void* k, const usv_strides* sk, const void* v,
+                        const usv_strides* sv, const int32_t* sel, const int32_t* k_per_head,
+                        int kmax, void* o, const usv_strides* so, float* o_f32, float* lse,
+                        float scale, int impl, void* ws, size_t ws_bytes, void* stream);
+
+/* Reads the device status word a kernel with bounded waits leaves in its workspace.
+ * Synchronises `stream`.  Returns USV_OK, USV_ERR_TIMEOUT or USV_ERR_CUDA. */
+int usv_workspace_status(const void* ws, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Token merge (Sec. 3.3, Eq. 6-14).
+ *   Partition: token (t,y,x) of the T x Hh x W raster grid is a destination iff
+ *   t % st == 0, y % sh == 0 and x % sw == 0 (the first token of its (st,sh,sw) block); every
+ *   other token is a source.
+ *   Plan (only when metric != NULL): head-averaged unit descriptors of `metric` (Eq. 7-8), best
+ *   destination j*(i) and cosine u_i per source over all destinations of the same batch element
+ *   (Eq. 9, ties to the lowest j), the r sources with the largest u are merged (Eq. 10-11, ties
+ *   to the lowest i).  The plan is written to dst_of / pos.
+ *   Apply: destinations become the mean of themselves and their merged sources (Eq. 12-13,
+ *   fp32 accumulation, bf16 RNE); output order is [unmerged sources ascending || destinations
+ *   ascending] (Eq. 14).
+ *
+ * x: bf16 [B,N,C] contiguous, N = T*Hh*W, C a multiple of 8.  x_merged: bf16 [B,N-r,C].
+ * metric: bf16 [B,N,Hm,dm] contiguous, dm in {64,128}; NULL = reuse the plan already stored in
+ *         dst_of/pos (lets one plan merge several tensors).
+ * r: number of sources merged per batch element, 0 <= r <= number of sources.
+ * dst_of: int32 [B,N], j*(i) for merged sources, -1 for every other token.
+ * pos: int32 [B,N], row of the merged sequence each original token reads back from.
+ * u_out, jstar_out: optional [B,N] (fp32 / int32): u_i and j*(i) for every source, (NaN,-1) at
+ *         destinations.  Only written when metric != NULL.
+ */
+size_t usv_token_merge_workspace(int B, int N, int C, int Hm, int dm);
+int usv_token_merge(int B, int N, int C, const void* x, int Hm, int dm, const void* metric, int T,
+                    int Hh, int W, int st, int sh, int sw, int r, void* x_merged, int32_t* dst_of,
+                    int32_t* pos, float* u_out, int32_t* jstar_out, void* ws, size_t ws_bytes,
+                    void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Token unmerge (Sec. 3.3, Eq. 15): y[b,n,:] = y_merged[b,pos[b,n],:].
+ * y_merged: bf16 [B,Nm,C]; pos: int32 [B,N] with entries in [0,Nm); y: bf16 [B,N,C] (written).
+ */
+int usv_token_unmerge(int B, int N, int Nm, int C, const void* y_merged, const int32_t* pos,
+                      void* y, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* USV_H_ */

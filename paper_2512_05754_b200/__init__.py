@@ -1,0 +1,10 @@
+"""B200-native (sm_100a) implementation of the USV sparsified attention hot path.
+
+Thin Python binding over the C-ABI library ``libusv.so`` (see ``include/usv.h``): argument
+marshalling only, every step of the path runs in the library's CUDA kernels.  PyTorch supplies
+device memory and streams.
+"""
+from .binding import (  # noqa: F401
+    USVError, lib, lib_path, block_scores, select_blocks, sparse_attn_fwd, token_merge,
+    token_unmerge, MergePlan, workspace_status, build_info, BLOCK,
+)

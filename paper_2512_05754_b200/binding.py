@@ -1,0 +1,227 @@
+"""ctypes binding of libusv.so.  Same names as the C entry points, torch tensors in and out."""
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+BLOCK = 64
+
+
+class USVError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        msg = "%s: %s (%s)" % (where, lib().usv_status_string(status).decode(),
+                               lib().usv_last_error().decode())
+        super().__init__(msg)
+
+
+class _Strides(ctypes.Structure):
+    _fields_ = [("sb", ctypes.c_int64), ("sh", ctypes.c_int64), ("sn", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def lib_path():
+    return _build.LIB
+
+
+def lib():
+    """Loads libusv.so (building it in-tree if it is missing and nvcc is available)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if not os.path.exists(path):
+        try:
+            _build.build()
+        except Exception as e:  # no silent fallback: the CUDA library is the product
+            raise ImportError("libusv.so is not built and could not be built: %s" % e)
+    L = ctypes.CDLL(path)
+    L.usv_status_string.restype = ctypes.c_char_p
+    L.usv_last_error.restype = ctypes.c_char_p
+    L.usv_build_info.restype = ctypes.c_char_p
+    for name in ("usv_block_scores_workspace", "usv_sparse_attn_workspace",
+                 "usv_token_merge_workspace"):
+        getattr(L, name).restype = ctypes.c_size_t
+    _lib = L
+    return L
+
+
+def build_info():
+    return lib().usv_build_info().decode()
+
+
+def _ptr(t):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream(device):
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def _check(status, where):
+    if status != 0:
+        raise USVError(status, where)
+
+
+def _view(t, name):
+    if t.dim() != 4 or t.dtype != torch.bfloat16 or not t.is_cuda or t.stride(3) != 1:
+        raise ValueError("%s must be a CUDA bf16 [B,H,N,d] view with a contiguous last axis" % name)
+    return _Strides(t.stride(0), t.stride(1), t.stride(2))
+
+
+_ws_cache = {}
+
+
+def _workspace(device, nbytes):
+    """Grow-only scratch buffer per (device, stream)."""
+    key = (device.index, torch.cuda.current_stream(device).cuda_stream)
+    buf = _ws_cache.get(key)
+    if buf is None or buf.numel() < nbytes:
+        buf = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+        _ws_cache[key] = buf
+    return buf
+
+
+def _k_array(k_per_head, H):
+    ks = [int(x) for x in k_per_head]
+    if len(ks) != H:
+        raise ValueError("k_per_head needs one entry per head")
+    return (ctypes.c_int32 * H)(*ks), max(ks)
+
+
+def block_scores(q, k, Nq=None, Nk=None, out=None):
+    """scores[b,h,I,J] of the pooled 64-token blocks; fp32 [B,H,NBq,NBk]."""
+    sq, sk = _view(q, "q"), _view(k, "k")
+    B, H, nq, d = q.shape
+    Nq = nq if Nq is None else int(Nq)
+    Nk = k.shape[2] if Nk is None else int(Nk)
+    NBq, NBk = (Nq + BLOCK - 1) // BLOCK, (Nk + BLOCK - 1) // BLOCK
+    if out is None:
+        out = torch.empty((B, H, NBq, NBk), dtype=torch.float32, device=q.device)
+    L = lib()
+    need = L.usv_block_scores_workspace(B, H, Nq, Nk, d)
+    ws = _workspace(q.device, need)
+    _check(L.usv_block_scores(B, H, Nq, Nk, d, _ptr(q), ctypes.byref(sq), _ptr(k),
+                              ctypes.byref(sk), _ptr(out), _ptr(ws), ctypes.c_size_t(ws.numel()),
+                              _stream(q.device)), "usv_block_scores")
+    return out
+
+
+def select_blocks(scores, k_per_head, kmax=None, out=None):
+    """Top-k key blocks per (b,h,I), ascending, ties to the lowest index; int32 [B,H,NBq,kmax]."""
+    if scores.dtype != torch.float32 or not scores.is_cuda or not scores.is_contiguous():
+        raise ValueError("scores must be a contiguous CUDA fp32 tensor")
+    B, H, NBq, NBk = scores.shape
+    karr, kmx = _k_array(k_per_head, H)
+    kmax = kmx if kmax is None else int(kmax)
+    if out is None:
+        out = torch.empty((B, H, NBq, kmax), dtype=torch.int32, device=scores.device)
+    _check(lib().usv_select_blocks(B, H, NBq, NBk, _ptr(scores), karr, kmax, _ptr(out),
+                                   _stream(scores.device)), "usv_select_blocks")
+    return out
+
+
+def sparse_attn_fwd(q, k, v, sel, k_per_head, N=None, scale=0.0, out=None, return_f32=False,
+                    return_lse=False, impl=0):
+    """Block-sparse attention forward.  Returns o (bf16, layout of q) and, if asked for, the
+    un-rounded fp32 output [B,H,N,d] and the log-sum-exp [B,H,N]."""
+    sq, sk, sv = _view(q, "q"), _view(k, "k"), _view(v, "v")
+    B, H, n, d = q.shape
+    N = n if N is None else int(N)
+    if sel.dtype != torch.int32 or not sel.is_contiguous() or not sel.is_cuda:
+        raise ValueError("sel must be a contiguous CUDA int32 tensor")
+    kmax = sel.shape[3]
+    karr, _ = _k_array(k_per_head, H)
+    if out is None:
+        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=q.device)
+    so = _view(out, "o")
+    o32 = torch.empty((B, H, N, d), dtype=torch.float32, device=q.device) if return_f32 else None
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if return_lse else None
+    L = lib()
+    need = L.usv_sparse_attn_workspace(B, H, N, d, kmax)
+    ws = _workspace(q.device, need)
+    _check(L.usv_sparse_attn_fwd(B, H, N, d, _ptr(q), ctypes.byref(sq), _ptr(k), ctypes.byref(sk),
+                                 _ptr(v), ctypes.byref(sv), _ptr(sel), karr, kmax, _ptr(out),
+                                 ctypes.byref(so), _ptr(o32), _ptr(lse), ctypes.c_float(scale),
+                                 int(impl), _ptr(ws), ctypes.c_size_t(ws.numel()),
+                                 _stream(q.device)), "usv_sparse_attn_fwd")
+    res = (out,)
+    if return_f32:
+        res += (o32,)
+    if return_lse:
+        res += (lse,)
+    return res if len(res) > 1 else out
+
+
+def workspace_status(device=None):
+    """Synchronises and returns the device status word of the current stream's workspace."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    ws = _workspace(device, 256)
+    return lib().usv_workspace_status(_ptr(ws), _stream(device))
+
+
+@dataclass
+class MergePlan:
+    dst_of: torch.Tensor                 # int32 [B,N]
+    pos: torch.Tensor                    # int32 [B,N]
+    grid: tuple
+    part: tuple
+    r: int
+    u: Optional[torch.Tensor] = None     # fp32 [B,N]
+    jstar: Optional[torch.Tensor] = None  # int32 [B,N]
+
+
+def token_merge(x, metric, grid, part, r, plan=None, debug=False):
+    """Merges x [B,N,C] (bf16).  With `metric` [B,N,Hm,dm] a new plan is computed; with
+    metric=None the given `plan` is applied.  Returns (x_merged [B,N-r,C], plan)."""
+    if x.dim() != 3 or x.dtype != torch.bfloat16 or not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x must be a contiguous CUDA bf16 [B,N,C] tensor")
+    B, N, C = x.shape
+    T, Hh, W = grid
+    st, sh, sw = part
+    dev = x.device
+    if metric is None:
+        if plan is None:
+            raise ValueError("either metric or plan is needed")
+        Hm = dm = 0
+        u = js = None
+    else:
+        if metric.dim() != 4 or metric.dtype != torch.bfloat16 or not metric.is_contiguous():
+            raise ValueError("metric must be a contiguous CUDA bf16 [B,N,Hm,dm] tensor")
+        Hm, dm = metric.shape[2], metric.shape[3]
+        plan = MergePlan(torch.empty((B, N), dtype=torch.int32, device=dev),
+                         torch.empty((B, N), dtype=torch.int32, device=dev), tuple(grid),
+                         tuple(part), int(r))
+        if debug:
+            plan.u = torch.empty((B, N), dtype=torch.float32, device=dev)
+            plan.jstar = torch.empty((B, N), dtype=torch.int32, device=dev)
+        u, js = plan.u, plan.jstar
+    out = torch.empty((B, max(N - r, 0), C), dtype=torch.bfloat16, device=dev)
+    L = lib()
+    need = L.usv_token_merge_workspace(B, N, C, Hm, dm if dm else 128)
+    ws = _workspace(dev, need)
+    _check(L.usv_token_merge(B, N, C, _ptr(x), Hm, dm, _ptr(metric), T, Hh, W, st, sh, sw, int(r),
+                             _ptr(out), _ptr(plan.dst_of), _ptr(plan.pos), _ptr(u), _ptr(js),
+                             _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(dev)),
+           "usv_token_merge")
+    return out, plan
+
+
+def token_unmerge(y_merged, pos, out=None):
+    """y[b,n,:] = y_merged[b,pos[b,n],:]."""
+    if (y_merged.dim() != 3 or y_merged.dtype != torch.bfloat16 or not y_merged.is_cuda
+            or not y_merged.is_contiguous()):
+        raise ValueError("y_merged must be a contiguous CUDA bf16 [B,Nm,C] tensor")
+    B, Nm, C = y_merged.shape
+    N = pos.shape[1]
+    if out is None:
+        out = torch.empty((B, N, C), dtype=torch.bfloat16, device=y_merged.device)
+    _check(lib().usv_token_unmerge(B, N, Nm, C, _ptr(y_merged), _ptr(pos), _ptr(out),
+                                   _stream(y_merged.device)), "usv_token_unmerge")
+    return out

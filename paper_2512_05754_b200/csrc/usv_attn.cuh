@@ -1,0 +1,23 @@
+// Argument block shared by the block-sparse attention kernels.
+#pragma once
+#include "usv_common.cuh"
+
+namespace usv {
+
+struct AttnArgs {
+    const __nv_bfloat16 *q, *k, *v;
+    __nv_bfloat16* o;
+    usv_strides sq, sk, sv, so;
+    const int32_t* sel;  // [B,H,NB,kmax]
+    float* o_f32;        // optional [B,H,N,D]
+    float* lse;          // optional [B,H,N]
+    unsigned int* status;  // optional device status word (bounded waits report here)
+    int B, H, N, NB, kmax;
+    float scale_log2;    // softmax scale * log2(e)
+    int k_per_head[USV_MAX_HEADS];
+    int head_order[USV_MAX_HEADS];  // heads sorted by descending k: heavy work is issued first
+};
+
+int launch_attn_mma(const AttnArgs& a, int d, cudaStream_t st);
+
+}  // namespace usv

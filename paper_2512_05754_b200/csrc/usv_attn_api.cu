@@ -1,0 +1,65 @@
+// Entry point of the block-sparse attention forward: validation, head ordering, dispatch.
+#include <algorithm>
+
+#include "usv_attn.cuh"
+
+extern "C" size_t usv_sparse_attn_workspace(int B, int H, int N, int d, int kmax) {
+    (void)B; (void)H; (void)N; (void)d; (void)kmax;
+    return 256;  // device status word (+ padding)
+}
+
+extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,
+                                   const void* k, const usv_strides* sk, const void* v,
+                                   const usv_strides* sv, const int32_t* sel,
+                                   const int32_t* k_per_head, int kmax, void* o,
+                                   const usv_strides* so, float* o_f32, float* lse, float scale,
+                                   int impl, void* ws, size_t ws_bytes, void* stream) {
+    using namespace usv;
+    if (B <= 0 || H <= 0 || N <= 0) return fail(USV_ERR_INVALID_ARG, "sparse_attn: B,H,N must be positive");
+    if (d != 64 && d != 128) return fail(USV_ERR_UNSUPPORTED, "sparse_attn: d=%d (need 64 or 128)", d);
+    if (H > USV_MAX_HEADS) return fail(USV_ERR_UNSUPPORTED, "sparse_attn: H > %d", USV_MAX_HEADS);
+    int rc;
+    if ((rc = check_view("q", q, sq, d)) != USV_OK) return rc;
+    if ((rc = check_view("k", k, sk, d)) != USV_OK) return rc;
+    if ((rc = check_view("v", v, sv, d)) != USV_OK) return rc;
+    if ((rc = check_view("o", o, so, d)) != USV_OK) return rc;
+    if (sel == nullptr || k_per_head == nullptr) return fail(USV_ERR_INVALID_ARG, "sparse_attn: null sel/k_per_head");
+    if (o_f32 != nullptr && !aligned16(o_f32)) return fail(USV_ERR_UNSUPPORTED, "sparse_attn: o_f32 misaligned");
+    if (!(scale >= 0.f)) return fail(USV_ERR_INVALID_ARG, "sparse_attn: scale must be >= 0");
+    if (impl != 0 && impl != 1) return fail(USV_ERR_INVALID_ARG, "sparse_attn: impl must be 0 or 1");
+    if (ws == nullptr) return fail(USV_ERR_INVALID_ARG, "sparse_attn: null workspace");
+    if (ws_bytes < usv_sparse_attn_workspace(B, H, N, d, kmax))
+        return fail(USV_ERR_WORKSPACE, "sparse_attn: workspace %zu < %zu", ws_bytes,
+                    usv_sparse_attn_workspace(B, H, N, d, kmax));
+    const int NB = ceil_div(N, USV_BLOCK);
+    AttnArgs a;
+    int kmx = 0;
+    for (int h = 0; h < H; ++h) {
+        if (k_per_head[h] < 1 || k_per_head[h] > NB)
+            return fail(USV_ERR_INVALID_ARG, "sparse_attn: k_per_head[%d]=%d outside [1,%d]", h,
+                        k_per_head[h], NB);
+        a.k_per_head[h] = k_per_head[h];
+        a.head_order[h] = h;
+        kmx = std::max(kmx, k_per_head[h]);
+    }
+    if (kmax < kmx) return fail(USV_ERR_INVALID_ARG, "sparse_attn: kmax=%d < max k=%d", kmax, kmx);
+    std::stable_sort(a.head_order, a.head_order + H,
+                     [&](int x, int y) { return k_per_head[x] > k_per_head[y]; });
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.k = static_cast<const __nv_bfloat16*>(k);
+    a.v = static_cast<const __nv_bfloat16*>(v);
+    a.o = static_cast<__nv_bfloat16*>(o);
+    a.sq = *sq; a.sk = *sk; a.sv = *sv; a.so = *so;
+    a.sel = sel;
+    a.o_f32 = o_f32;
+    a.lse = lse;
+    a.status = static_cast<unsigned int*>(ws);
+    a.B = B; a.H = H; a.N = N; a.NB = NB; a.kmax = kmax;
+    const float sc = scale == 0.f ? 1.0f / sqrtf((float)d) : scale;
+    a.scale_log2 = sc * 1.4426950408889634f;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(ws, 0, 256, st);
+    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: memset: %s", cudaGetErrorString(e));
+    (void)impl;
+    return launch_attn_mma(a, d, st);
+}

@@ -1,0 +1,590 @@
+// Token merge / unmerge (Sec. 3.3 of the USV paper).
+//
+//   desc_kernel        Eq. 7-8   head-averaged, unit-normalised key descriptors (HBM stream)
+//   src_list_kernel    Eq. 6     ascending list of source tokens of the bipartite partition
+//   match_kernel       Eq. 8-9   cosine of every source against every destination of its batch
+//                                element with a fused row arg-max (fp32 CUDA cores; the result
+//                                decides an integer that is compared with an fp64 evaluation)
+//   plan_kernel        Eq. 10-11, 14  radix-select of the r most confident sources, ordered
+//                                compaction, dst_of / pos
+//   csr_* kernels      Eq. 12    sources grouped by destination
+//   merge_kernel       Eq. 13-14 warp-per-row gather + mean, 16-byte accesses
+//   unmerge_kernel     Eq. 15    warp-per-row gather copy, 16-byte accesses
+#include <math.h>
+
+#include "usv_common.cuh"
+
+namespace usv {
+
+struct Part {
+    int T, Hh, W, st, sh, sw;
+    int nHy, nWx, nB;  // destinations per axis (y, x) and in total
+    __host__ __device__ bool is_dst(int n) const {
+        const int x = n % W, y = (n / W) % Hh, t = n / (W * Hh);
+        return (t % st == 0) && (y % sh == 0) && (x % sw == 0);
+    }
+    // ordinal (ascending token order) of a destination token
+    __host__ __device__ int ord(int n) const {
+        const int x = n % W, y = (n / W) % Hh, t = n / (W * Hh);
+        return ((t / st) * nHy + y / sh) * nWx + x / sw;
+    }
+    __host__ __device__ int dst_token(int o) const {
+        const int dx = o % nWx, dy = (o / nWx) % nHy, dt = o / (nWx * nHy);
+        return ((dt * st) * Hh + dy * sh) * W + dx * sw;
+    }
+};
+
+// ---------------------------------------------------------------------------- descriptors
+// One warp per token.  DM/8 lanes cover one head's row with 16-byte loads; 32/(DM/8) heads are
+// read in parallel and combined with shuffles.
+template <int DM>
+__global__ void __launch_bounds__(256) desc_kernel(const __nv_bfloat16* __restrict__ metric,
+                                                   float* __restrict__ mhat, int64_t tokens,
+                                                   int Hm) {
+    constexpr int LPH = DM / 8;    // lanes per head row
+    constexpr int HPW = 32 / LPH;  // heads handled at once
+    const int64_t tok = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (tok >= tokens) return;
+    const int lane = threadIdx.x & 31;
+    const int chunk = lane % LPH, hsub = lane / LPH;
+    const __nv_bfloat16* src = metric + tok * Hm * DM + chunk * 8;
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int h = hsub; h < Hm; h += HPW) {
+        float f[8];
+        bf16x8_to_float(__ldg(reinterpret_cast<const uint4*>(src + (int64_t)h * DM)), f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] += f[e];
+    }
+#pragma unroll
+    for (int o = LPH; o < 32; o <<= 1)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+    float n2 = 0.f;
+    const float invH = 1.0f / (float)Hm;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        acc[e] *= invH;
+        n2 = fmaf(acc[e], acc[e], n2);
+    }
+#pragma unroll
+    for (int o = 1; o < LPH; o <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+    const float inv = 1.0f / fmaxf(sqrtf(n2), 1e-12f);
+    if (hsub == 0) {
+        float* dst = mhat + tok * DM + chunk * 8;
+        *reinterpret_cast<float4*>(dst) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+        *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[4] * inv, acc[5] * inv, acc[6] * inv, acc[7] * inv);
+    }
+}
+
+// ---------------------------------------------------------------------------- block scan (1024)
+__device__ __forceinline__ int block_scan_1024(int v, int* scratch, int* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int incl = warp_incl_scan(v);
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const int w = scratch[lane];
+        const int wi = warp_incl_scan(w);
+        scratch[lane] = wi - w;
+        if (lane == 31) scratch[32] = wi;
+    }
+    __syncthreads();
+    const int res = scratch[warp] + incl - v;
+    *total = scratch[32];
+    __syncthreads();
+    return res;
+}
+
+// Ascending list of the source tokens (same for every batch element).  One CTA, 1024 threads.
+__global__ void __launch_bounds__(1024) src_list_kernel(Part p, int N, int32_t* __restrict__ src_idx) {
+    __shared__ int scratch[33];
+    int base = 0;
+    for (int n0 = 0; n0 < N; n0 += 1024) {
+        const int n = n0 + threadIdx.x;
+        const int flag = (n < N && !p.is_dst(n)) ? 1 : 0;
+        int tot;
+        const int r = base + block_scan_1024(flag, scratch, &tot);
+        if (flag) src_idx[r] = n;
+        base += tot;
+    }
+}
+
+// ---------------------------------------------------------------------------- matching
+// CTA: 256 threads, 64 sources x (all destinations in tiles of 64).  The 64 source descriptors
+// stay in shared memory for the whole sweep; destination tiles stream through in chunks of 32
+// features.  Each thread keeps the running best of its 4 rows over its 4 columns per tile;
+// columns are visited in ascending destination order and replaced only on strict improvement, so
+// equal cosines resolve to the lowest destination.
+template <int DM>
+__global__ void __launch_bounds__(256) match_kernel(const float* __restrict__ mhat, Part p, int N,
+                                                    int nA, const int32_t* __restrict__ src_idx,
+                                                    int32_t* __restrict__ jstar_s,
+                                                    float* __restrict__ u_s) {
+    constexpr int TK = 32;
+    __shared__ __align__(16) float As[DM][64 + 4];
+    __shared__ __align__(16) float Bs[TK][64 + 4];
+    const int b = blockIdx.y;
+    const int a0 = blockIdx.x * 64;
+    const float* M = mhat + (int64_t)b * N * DM;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+
+    for (int idx = threadIdx.x; idx < 64 * (DM / 4); idx += 256) {
+        const int r = idx / (DM / 4), c4 = idx % (DM / 4);
+        float4 v = make_float4(0, 0, 0, 0);
+        if (a0 + r < nA) v = *reinterpret_cast<const float4*>(M + (int64_t)src_idx[a0 + r] * DM + c4 * 4);
+        As[c4 * 4 + 0][r] = v.x; As[c4 * 4 + 1][r] = v.y;
+        As[c4 * 4 + 2][r] = v.z; As[c4 * 4 + 3][r] = v.w;
+    }
+    float best[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    int besti[4] = {0x7fffffff, 0x7fffffff, 0x7fffffff, 0x7fffffff};
+    __syncthreads();
+
+    for (int j0 = 0; j0 < p.nB; j0 += 64) {
+        float acc[4][4] = {};
+        for (int k0 = 0; k0 < DM; k0 += TK) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int idx = threadIdx.x + t * 256;
+                const int r = idx / 8, c4 = idx % 8;
+                float4 v = make_float4(0, 0, 0, 0);
+                if (j0 + r < p.nB)
+                    v = *reinterpret_cast<const float4*>(M + (int64_t)p.dst_token(j0 + r) * DM + k0 + c4 * 4);
+                Bs[c4 * 4 + 0][r] = v.x; Bs[c4 * 4 + 1][r] = v.y;
+                Bs[c4 * 4 + 2][r] = v.z; Bs[c4 * 4 + 3][r] = v.w;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int e = 0; e < TK; ++e) {
+                const float4 av = *reinterpret_cast<const float4*>(&As[k0 + e][ty * 4]);
+                const float4 bv = *reinterpret_cast<const float4*>(&Bs[e][tx * 4]);
+                const float ar[4] = {av.x, av.y, av.z, av.w};
+                const float br[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(ar[i], br[j], acc[i][j]);
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int o = j0 + tx * 4 + j;
+            if (o < p.nB) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (acc[i][j] > best[i]) {
+                        best[i] = acc[i][j];
+                        besti[i] = o;
+                    }
+            }
+        }
+    }
+    // combine the 16 threads (consecutive lanes) that share a row
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll
+        for (int o = 1; o < 16; o <<= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best[i], o);
+            const int oi = __shfl_xor_sync(0xffffffffu, besti[i], o);
+            if (ov > best[i] || (ov == best[i] && oi < besti[i])) {
+                best[i] = ov;
+                besti[i] = oi;
+            }
+        }
+        const int a = a0 + ty * 4 + i;
+        if (tx == 0 && a < nA) {
+            jstar_s[(int64_t)b * nA + a] = p.dst_token(besti[i]);
+            u_s[(int64_t)b * nA + a] = best[i];
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------- plan
+// One CTA (1024 threads) per batch element.  Radix-select of the r-th largest u, then an ordered
+// pass that marks the merged sources (ties to the lowest source index) and writes dst_of / pos.
+__global__ void __launch_bounds__(1024) plan_kernel(Part p, int N, int nA, int r,
+                                                    const int32_t* __restrict__ src_idx,
+                                                    const int32_t* __restrict__ jstar_s,
+                                                    const float* __restrict__ u_s,
+                                                    int32_t* __restrict__ dst_of,
+                                                    int32_t* __restrict__ pos,
+                                                    float* __restrict__ u_out,
+                                                    int32_t* __restrict__ jstar_out) {
+    __shared__ int hist[256];
+    __shared__ int scratch[33];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_remaining;
+    const int b = blockIdx.x;
+    const float* u = u_s + (int64_t)b * nA;
+    const int32_t* js = jstar_s + (int64_t)b * nA;
+    int32_t* d_of = dst_of + (int64_t)b * N;
+    int32_t* ps = pos + (int64_t)b * N;
+    const int nU = nA - r;
+
+    uint32_t T = 0xffffffffu;  // r == 0: nothing is above or equal (need_eq = 0 below)
+    int need_eq = 0;
+    if (r > 0) {
+        if (threadIdx.x == 0) {
+            s_prefix = 0;
+            s_remaining = r;
+        }
+        __syncthreads();
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+            __syncthreads();
+            const uint32_t prefix = s_prefix;
+            const uint32_t mask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
+            for (int a = threadIdx.x; a < nA; a += 1024) {
+                const uint32_t key = float_key(u[a]);
+                if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+            }
+            __syncthreads();
+            if (threadIdx.x < 32) {
+                const int lane = threadIdx.x;
+                const int remaining = s_remaining;
+                int local[8], sum = 0;
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    local[t] = hist[255 - (lane * 8 + t)];
+                    sum += local[t];
+                }
+                const int incl = warp_incl_scan(sum);
+                int before = incl - sum;
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    if (before < remaining && remaining <= before + local[t]) {
+                        s_prefix = prefix | ((uint32_t)(255 - (lane * 8 + t)) << shift);
+                        s_remaining = remaining - before;
+                    }
+                    before += local[t];
+                }
+            }
+            __syncthreads();
+        }
+        T = s_prefix;
+        need_eq = s_remaining;
+    }
+
+    int base_eq = 0, base_un = 0;
+    for (int a0 = 0; a0 < nA; a0 += 1024) {
+        const int a = a0 + threadIdx.x;
+        const bool in = a < nA;
+        const float ua = in ? u[a] : 0.f;
+        const uint32_t key = in ? float_key(ua) : 0u;
+        const int is_gt = (in && r > 0 && key > T) ? 1 : 0;
+        const int is_eq = (in && r > 0 && key == T) ? 1 : 0;
+        int tot_eq, tot_un;
+        const int eq_rank = base_eq + block_scan_1024(is_eq, scratch, &tot_eq);
+        const int merged = is_gt | (is_eq && eq_rank < need_eq);
+        const int un = (in && !merged) ? 1 : 0;
+        const int un_rank = base_un + block_scan_1024(un, scratch, &tot_un);
+        if (in) {
+            const int n = src_idx[a];
+            const int j = js[a];
+            if (merged) {
+                d_of[n] = j;
+                ps[n] = nU + p.ord(j);
+            } else {
+                d_of[n] = -1;
+                ps[n] = un_rank;
+            }
+            if (u_out) u_out[(int64_t)b * N + n] = ua;
+            if (jstar_out) jstar_out[(int64_t)b * N + n] = j;
+        }
+        base_eq += tot_eq;
+        base_un += tot_un;
+    }
+    for (int o = threadIdx.x; o < p.nB; o += 1024) {
+        const int n = p.dst_token(o);
+        d_of[n] = -1;
+        ps[n] = nU + o;
+        if (u_out) u_out[(int64_t)b * N + n] = __int_as_float(0x7fc00000);
+        if (jstar_out) jstar_out[(int64_t)b * N + n] = -1;
+    }
+}
+
+// ---------------------------------------------------------------------------- CSR of M(j)
+__global__ void __launch_bounds__(256) csr_count_kernel(Part p, int N, int nU,
+                                                        const int32_t* __restrict__ dst_of,
+                                                        const int32_t* __restrict__ pos,
+                                                        int32_t* __restrict__ cnt,
+                                                        int32_t* __restrict__ row_src) {
+    const int b = blockIdx.y;
+    const int n = blockIdx.x * 256 + threadIdx.x;
+    if (n >= N) return;
+    const int j = dst_of[(int64_t)b * N + n];
+    if (j >= 0) atomicAdd(&cnt[(int64_t)b * p.nB + p.ord(j)], 1);
+    else if (!p.is_dst(n)) row_src[(int64_t)b * nU + pos[(int64_t)b * N + n]] = n;
+}
+
+// exclusive scan of cnt[b,:] -> off[b,0..nB], cursor[b,:] = off[b,:nB].  One CTA per batch element.
+__global__ void __launch_bounds__(1024) csr_scan_kernel(int nB, const int32_t* __restrict__ cnt,
+                                                        int32_t* __restrict__ off,
+                                                        int32_t* __restrict__ cursor) {
+    __shared__ int scratch[33];
+    const int b = blockIdx.x;
+    int base = 0;
+    for (int o0 = 0; o0 < nB; o0 += 1024) {
+        const int o = o0 + threadIdx.x;
+        const int c = o < nB ? cnt[(int64_t)b * nB + o] : 0;
+        int tot;
+        const int e = base + block_scan_1024(c, scratch, &tot);
+        if (o < nB) {
+            off[(int64_t)b * (nB + 1) + o] = e;
+            cursor[(int64_t)b * nB + o] = e;
+        }
+        base += tot;
+    }
+    if (threadIdx.x == 0) off[(int64_t)b * (nB + 1) + nB] = base;
+}
+
+__global__ void __launch_bounds__(256) csr_fill_kernel(Part p, int N, int r,
+                                                       const int32_t* __restrict__ dst_of,
+                                                       int32_t* __restrict__ cursor,
+                                                       int32_t* __restrict__ csr) {
+    const int b = blockIdx.y;
+    const int n = blockIdx.x * 256 + threadIdx.x;
+    if (n >= N) return;
+    const int j = dst_of[(int64_t)b * N + n];
+    if (j >= 0) {
+        const int slot = atomicAdd(&cursor[(int64_t)b * p.nB + p.ord(j)], 1);
+        csr[(int64_t)b * r + slot] = n;
+    }
+}
+
+// ---------------------------------------------------------------------------- merge
+// One warp per output row.  Rows [0,nU) copy an unmerged source; rows [nU, nU+nB) hold a
+// destination averaged with its merged sources, summed in ascending source index.
+__global__ void __launch_bounds__(256) merge_kernel(Part p, int N, int C, int nU, int Nm, int r,
+                                                    const __nv_bfloat16* __restrict__ x,
+                                                    const int32_t* __restrict__ row_src,
+                                                    const int32_t* __restrict__ off,
+                                                    int32_t* __restrict__ csr,
+                                                    __nv_bfloat16* __restrict__ out, int64_t rows) {
+    const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (gw >= rows) return;
+    const int lane = threadIdx.x & 31;
+    const int b = (int)(gw / Nm), row = (int)(gw % Nm);
+    const __nv_bfloat16* xb = x + (int64_t)b * N * C;
+    uint4* dst = reinterpret_cast<uint4*>(out + ((int64_t)b * Nm + row) * C);
+    const int nvec = C / 8;
+    if (row < nU) {
+        const uint4* src = reinterpret_cast<const uint4*>(xb + (int64_t)row_src[(int64_t)b * nU + row] * C);
+        for (int c = lane; c < nvec; c += 32) dst[c] = __ldg(src + c);
+        return;
+    }
+    const int o = row - nU;
+    const int j = p.dst_token(o);
+    const int beg = off[(int64_t)b * (p.nB + 1) + o], end = off[(int64_t)b * (p.nB + 1) + o + 1];
+    const int len = end - beg;
+    int32_t* list = csr + (int64_t)b * r + beg;
+    const uint4* srcj = reinterpret_cast<const uint4*>(xb + (int64_t)j * C);
+    if (len == 0) {
+        for (int c = lane; c < nvec; c += 32) dst[c] = __ldg(srcj + c);
+        return;
+    }
+    int myid = 0x7fffffff;
+    if (len <= 32) {
+        // rank sort in registers: lane s ends up holding the s-th smallest source index
+        const int id = lane < len ? list[lane] : 0x7fffffff;
+        int rank = 0;
+#pragma unroll
+        for (int s = 0; s < 32; ++s) {
+            const int other = __shfl_sync(0xffffffffu, id, s);
+            rank += (other < id) ? 1 : 0;
+        }
+        // ids are distinct, so ranks of the valid lanes are a permutation of 0..len-1
+#pragma unroll
+        for (int s = 0; s < 32; ++s) {
+            const int oid = __shfl_sync(0xffffffffu, id, s);
+            const int orank = __shfl_sync(0xffffffffu, rank, s);
+            if (orank == lane && s < len) myid = oid;
+        }
+    } else {
+        // rare long list: in-place selection sort of the segment by this warp
+        for (int s = 0; s < len - 1; ++s) {
+            int bestv = 0x7fffffff, bestp = -1;
+            for (int t = s + lane; t < len; t += 32) {
+                const int v = list[t];
+                if (v < bestv) { bestv = v; bestp = t; }
+            }
+#pragma unroll
+            for (int w = 16; w > 0; w >>= 1) {
+                const int ov = __shfl_xor_sync(0xffffffffu, bestv, w);
+                const int op = __shfl_xor_sync(0xffffffffu, bestp, w);
+                if (ov < bestv) { bestv = ov; bestp = op; }
+            }
+            if (lane == 0 && bestp != s) {
+                const int tmp = list[s];
+                list[s] = bestv;
+                list[bestp] = tmp;
+            }
+            __syncwarp();
+        }
+    }
+    const float inv = 1.0f / (float)(len + 1);
+    for (int c0 = 0; c0 < nvec; c0 += 32) {
+        const int c = c0 + lane;
+        const bool act = c < nvec;
+        float acc[8];
+        if (act) bf16x8_to_float(__ldg(srcj + c), acc);
+        for (int s = 0; s < len; ++s) {
+            const int i = len <= 32 ? __shfl_sync(0xffffffffu, myid, s) : list[s];
+            if (act) {
+                float f[8];
+                bf16x8_to_float(__ldg(reinterpret_cast<const uint4*>(xb + (int64_t)i * C) + c), f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] += f[e];
+            }
+        }
+        if (act) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] *= inv;
+            dst[c] = float8_to_bf16x8(acc);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------- unmerge
+__global__ void __launch_bounds__(256) unmerge_kernel(int N, int Nm, int C,
+                                                      const __nv_bfloat16* __restrict__ ym,
+                                                      const int32_t* __restrict__ pos,
+                                                      __nv_bfloat16* __restrict__ y, int64_t rows) {
+    const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (gw >= rows) return;
+    const int lane = threadIdx.x & 31;
+    const int b = (int)(gw / N);
+    const int pr = pos[gw];
+    const uint4* src = reinterpret_cast<const uint4*>(ym + ((int64_t)b * Nm + pr) * C);
+    uint4* dst = reinterpret_cast<uint4*>(y + gw * C);
+    const int nvec = C / 8;
+    for (int c = lane; c < nvec; c += 32) dst[c] = __ldg(src + c);
+}
+
+// ---------------------------------------------------------------------------- host side
+struct MergeWs {
+    size_t mhat, src_idx, jstar_s, u_s, row_src, cnt, off, cursor, csr, total;
+};
+
+static MergeWs merge_layout(int B, int N, int dm, int nA, int nB) {
+    MergeWs w;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    w.mhat = take((size_t)B * N * (dm > 0 ? dm : 1) * sizeof(float));
+    w.src_idx = take((size_t)nA * 4);
+    w.jstar_s = take((size_t)B * nA * 4);
+    w.u_s = take((size_t)B * nA * 4);
+    w.row_src = take((size_t)B * nA * 4);
+    w.cnt = take((size_t)B * nB * 4);
+    w.off = take((size_t)B * (nB + 1) * 4);
+    w.cursor = take((size_t)B * nB * 4);
+    w.csr = take((size_t)B * nA * 4);
+    w.total = o;
+    return w;
+}
+
+}  // namespace usv
+
+extern "C" size_t usv_token_merge_workspace(int B, int N, int C, int Hm, int dm) {
+    (void)C; (void)Hm;
+    if (B <= 0 || N <= 0) return 0;
+    // sized for the worst partition (every token but one is a source / a destination)
+    return usv::merge_layout(B, N, dm, N, N).total;
+}
+
+extern "C" int usv_token_merge(int B, int N, int C, const void* x, int Hm, int dm,
+                               const void* metric, int T, int Hh, int W, int st, int sh, int sw,
+                               int r, void* x_merged, int32_t* dst_of, int32_t* pos, float* u_out,
+                               int32_t* jstar_out, void* ws, size_t ws_bytes, void* stream) {
+    using namespace usv;
+    if (B <= 0 || N <= 0 || C <= 0) return fail(USV_ERR_INVALID_ARG, "token_merge: B,N,C must be positive");
+    if (T <= 0 || Hh <= 0 || W <= 0 || (int64_t)T * Hh * W != N)
+        return fail(USV_ERR_INVALID_ARG, "token_merge: T*Hh*W = %lld != N = %d", (long long)T * Hh * W, N);
+    if (st <= 0 || sh <= 0 || sw <= 0) return fail(USV_ERR_INVALID_ARG, "token_merge: partition sizes must be positive");
+    if (C % 8) return fail(USV_ERR_UNSUPPORTED, "token_merge: C=%d not a multiple of 8", C);
+    if (x == nullptr || x_merged == nullptr || dst_of == nullptr || pos == nullptr || ws == nullptr)
+        return fail(USV_ERR_INVALID_ARG, "token_merge: null pointer");
+    if (!aligned16(x) || !aligned16(x_merged) || !aligned16(ws))
+        return fail(USV_ERR_UNSUPPORTED, "token_merge: x/x_merged/ws not 16-byte aligned");
+    Part p;
+    p.T = T; p.Hh = Hh; p.W = W; p.st = st; p.sh = sh; p.sw = sw;
+    p.nHy = ceil_div(Hh, sh); p.nWx = ceil_div(W, sw);
+    p.nB = ceil_div(T, st) * p.nHy * p.nWx;
+    const int nA = N - p.nB;
+    if (r < 0 || r > nA) return fail(USV_ERR_INVALID_ARG, "token_merge: r=%d outside [0,%d] (number of sources)", r, nA);
+    if (metric != nullptr) {
+        if (dm != 64 && dm != 128) return fail(USV_ERR_UNSUPPORTED, "token_merge: dm=%d (need 64 or 128)", dm);
+        if (Hm <= 0) return fail(USV_ERR_INVALID_ARG, "token_merge: Hm must be positive");
+        if (!aligned16(metric)) return fail(USV_ERR_UNSUPPORTED, "token_merge: metric not 16-byte aligned");
+    }
+    if ((int64_t)B > 65535) return fail(USV_ERR_UNSUPPORTED, "token_merge: B > 65535");
+    if (ws_bytes < usv_token_merge_workspace(B, N, C, Hm, dm))
+        return fail(USV_ERR_WORKSPACE, "token_merge: workspace %zu < %zu", ws_bytes,
+                    usv_token_merge_workspace(B, N, C, Hm, dm));
+    const MergeWs L = merge_layout(B, N, dm, nA, p.nB);
+    char* base = static_cast<char*>(ws);
+    float* mhat = reinterpret_cast<float*>(base + L.mhat);
+    int32_t* src_idx = reinterpret_cast<int32_t*>(base + L.src_idx);
+    int32_t* jstar_s = reinterpret_cast<int32_t*>(base + L.jstar_s);
+    float* u_s = reinterpret_cast<float*>(base + L.u_s);
+    int32_t* row_src = reinterpret_cast<int32_t*>(base + L.row_src);
+    int32_t* cnt = reinterpret_cast<int32_t*>(base + L.cnt);
+    int32_t* off = reinterpret_cast<int32_t*>(base + L.off);
+    int32_t* cursor = reinterpret_cast<int32_t*>(base + L.cursor);
+    int32_t* csr = reinterpret_cast<int32_t*>(base + L.csr);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int nU = nA - r, Nm = N - r;
+
+    if (metric != nullptr) {
+        const int64_t tokens = (int64_t)B * N;
+        const unsigned dg = (unsigned)((tokens + 7) / 8);
+        if (dm == 128) desc_kernel<128><<<dg, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(metric), mhat, tokens, Hm);
+        else desc_kernel<64><<<dg, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(metric), mhat, tokens, Hm);
+        USV_CHECK_LAUNCH("desc_kernel");
+        if (nA > 0) {
+            src_list_kernel<<<1, 1024, 0, s>>>(p, N, src_idx);
+            USV_CHECK_LAUNCH("src_list_kernel");
+            dim3 mg(ceil_div(nA, 64), B);
+            if (dm == 128) match_kernel<128><<<mg, 256, 0, s>>>(mhat, p, N, nA, src_idx, jstar_s, u_s);
+            else match_kernel<64><<<mg, 256, 0, s>>>(mhat, p, N, nA, src_idx, jstar_s, u_s);
+            USV_CHECK_LAUNCH("match_kernel");
+        }
+        plan_kernel<<<B, 1024, 0, s>>>(p, N, nA, r, src_idx, jstar_s, u_s, dst_of, pos, u_out, jstar_out);
+        USV_CHECK_LAUNCH("plan_kernel");
+    }
+    cudaError_t e = cudaMemsetAsync(cnt, 0, (size_t)B * p.nB * 4, s);
+    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: memset: %s", cudaGetErrorString(e));
+    dim3 tg(ceil_div(N, 256), B);
+    csr_count_kernel<<<tg, 256, 0, s>>>(p, N, nU, dst_of, pos, cnt, row_src);
+    USV_CHECK_LAUNCH("csr_count_kernel");
+    csr_scan_kernel<<<B, 1024, 0, s>>>(p.nB, cnt, off, cursor);
+    USV_CHECK_LAUNCH("csr_scan_kernel");
+    if (r > 0) {
+        csr_fill_kernel<<<tg, 256, 0, s>>>(p, N, r, dst_of, cursor, csr);
+        USV_CHECK_LAUNCH("csr_fill_kernel");
+    }
+    const int64_t rows = (int64_t)B * Nm;
+    merge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, s>>>(
+        p, N, C, nU, Nm, r, static_cast<const __nv_bfloat16*>(x), row_src, off, csr,
+        static_cast<__nv_bfloat16*>(x_merged), rows);
+    USV_CHECK_LAUNCH("merge_kernel");
+    return USV_OK;
+}
+
+extern "C" int usv_token_unmerge(int B, int N, int Nm, int C, const void* y_merged,
+                                 const int32_t* pos, void* y, void* stream) {
+    using namespace usv;
+    if (B <= 0 || N <= 0 || Nm <= 0 || C <= 0 || Nm > N)
+        return fail(USV_ERR_INVALID_ARG, "token_unmerge: need B,N,Nm,C > 0 and Nm <= N");
+    if (C % 8) return fail(USV_ERR_UNSUPPORTED, "token_unmerge: C=%d not a multiple of 8", C);
+    if (y_merged == nullptr || pos == nullptr || y == nullptr)
+        return fail(USV_ERR_INVALID_ARG, "token_unmerge: null pointer");
+    if (!aligned16(y_merged) || !aligned16(y))
+        return fail(USV_ERR_UNSUPPORTED, "token_unmerge: y_merged/y not 16-byte aligned");
+    const int64_t rows = (int64_t)B * N;
+    unmerge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        N, Nm, C, static_cast<const __nv_bfloat16*>(y_merged), pos,
+        static_cast<__nv_bfloat16*>(y), rows);
+    USV_CHECK_LAUNCH("unmerge_kernel");
+    return USV_OK;
+}

@@ -1,0 +1,175 @@
+// Coarse stage of the key-block selection: block pooling (HBM stream) and block scores.
+//
+//   pool_kernel   : one CTA per (tensor, b, h, block); 16-byte loads, eight rows in flight per
+//                   thread, fp32 tree reduction, mean over the VALID rows of the block.
+//   scores_kernel : fp32 CUDA-core NT GEMM per (b,h), 64x64 output tile, 4x4 per thread.
+//                   Kept in fp32 (not bf16 tensor cores) because the result decides an integer
+//                   (the top-k set) that is compared with an fp64 evaluation.
+#include "usv_common.cuh"
+
+namespace usv {
+
+struct PoolArgs {
+    const __nv_bfloat16* x[2];
+    int64_t sb[2], sh[2], sn[2];
+    int N[2], NB[2];
+    float* out[2];  // [B,H,NB,d]
+    int H;
+};
+
+// D = head dim (64 or 128).  Threads: 128.  A row of D bf16 is D/8 uint4; TPR threads per row.
+template <int D>
+__global__ void __launch_bounds__(128) pool_kernel(const PoolArgs a) {
+    constexpr int TPR = D / 8;          // 16 (d=128) or 8 (d=64)
+    constexpr int RPI = 128 / TPR;      // rows per iteration: 8 or 16
+    constexpr int ITERS = USV_BLOCK / RPI;
+    const int which = blockIdx.z;
+    const int NB = a.NB[which];
+    const int I = blockIdx.x;
+    if (I >= NB) return;
+    const int bh = blockIdx.y;
+    const int b = bh / a.H, h = bh % a.H;
+    const int N = a.N[which];
+    const int col = threadIdx.x % TPR, rg = threadIdx.x / TPR;
+    const __nv_bfloat16* base =
+        a.x[which] + b * a.sb[which] + h * a.sh[which] + (int64_t)col * 8;
+    const int64_t sn = a.sn[which];
+    const int row0 = I * USV_BLOCK;
+    const int nvalid = min(USV_BLOCK, N - row0);
+
+    uint4 v[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        const int r = it * RPI + rg;
+        v[it] = make_uint4(0, 0, 0, 0);
+        if (r < nvalid) v[it] = __ldg(reinterpret_cast<const uint4*>(base + (row0 + r) * sn));
+    }
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        float f[8];
+        bf16x8_to_float(v[it], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] += f[e];
+    }
+    __shared__ float red[RPI][D + 4];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) red[rg][col * 8 + e] = acc[e];
+    __syncthreads();
+    if (threadIdx.x < D) {
+        float s = 0.f;
+#pragma unroll
+        for (int g = 0; g < RPI; ++g) s += red[g][threadIdx.x];
+        a.out[which][((int64_t)bh * NB + I) * D + threadIdx.x] = s / (float)nvalid;
+    }
+}
+
+// scores[bh, I, J] = scale * sum_e qbar[bh,I,e] * kbar[bh,J,e]
+// CTA: 256 threads, 64x64 tile; smem tiles stored e-major so that the inner product reads
+// float4 along the tile row/column.
+__global__ void __launch_bounds__(256) scores_kernel(const float* __restrict__ qbar,
+                                                     const float* __restrict__ kbar,
+                                                     float* __restrict__ scores, int NBq, int NBk,
+                                                     int d, float scale) {
+    constexpr int TM = 64, TN = 64, TK = 32;
+    __shared__ __align__(16) float As[TK][TM + 4];
+    __shared__ __align__(16) float Bs[TK][TN + 4];
+    const int bh = blockIdx.z;
+    const int i0 = blockIdx.y * TM, j0 = blockIdx.x * TN;
+    const float* A = qbar + (int64_t)bh * NBq * d;
+    const float* Bm = kbar + (int64_t)bh * NBk * d;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < d; k0 += TK) {
+        // 64 rows x 32 floats = 512 float4; 256 threads -> 2 each
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const int idx = threadIdx.x + t * 256;
+            const int r = idx / 8, c4 = idx % 8;
+            float4 va = make_float4(0, 0, 0, 0), vb = va;
+            if (i0 + r < NBq)
+                va = *reinterpret_cast<const float4*>(A + (int64_t)(i0 + r) * d + k0 + c4 * 4);
+            if (j0 + r < NBk)
+                vb = *reinterpret_cast<const float4*>(Bm + (int64_t)(j0 + r) * d + k0 + c4 * 4);
+            As[c4 * 4 + 0][r] = va.x; As[c4 * 4 + 1][r] = va.y;
+            As[c4 * 4 + 2][r] = va.z; As[c4 * 4 + 3][r] = va.w;
+            Bs[c4 * 4 + 0][r] = vb.x; Bs[c4 * 4 + 1][r] = vb.y;
+            Bs[c4 * 4 + 2][r] = vb.z; Bs[c4 * 4 + 3][r] = vb.w;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < TK; ++e) {
+            const float4 av = *reinterpret_cast<const float4*>(&As[e][ty * 4]);
+            const float4 bv = *reinterpret_cast<const float4*>(&Bs[e][tx * 4]);
+            const float ar[4] = {av.x, av.y, av.z, av.w};
+            const float br[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(ar[i], br[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    float* out = scores + (int64_t)bh * NBq * NBk;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int I = i0 + ty * 4 + i;
+        if (I >= NBq) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int J = j0 + tx * 4 + j;
+            if (J < NBk) out[(int64_t)I * NBk + J] = acc[i][j] * scale;
+        }
+    }
+}
+
+}  // namespace usv
+
+extern "C" size_t usv_block_scores_workspace(int B, int H, int Nq, int Nk, int d) {
+    if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || d <= 0) return 0;
+    const size_t nbq = usv::ceil_div(Nq, USV_BLOCK), nbk = usv::ceil_div(Nk, USV_BLOCK);
+    return usv::align_up((size_t)B * H * nbq * d * sizeof(float), 256) +
+           usv::align_up((size_t)B * H * nbk * d * sizeof(float), 256);
+}
+
+extern "C" int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void* q,
+                                const usv_strides* sq, const void* k, const usv_strides* sk,
+                                float* scores, void* ws, size_t ws_bytes, void* stream) {
+    using namespace usv;
+    if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0)
+        return fail(USV_ERR_INVALID_ARG, "block_scores: B,H,Nq,Nk must be positive");
+    if (d != 64 && d != 128) return fail(USV_ERR_UNSUPPORTED, "block_scores: d=%d (need 64 or 128)", d);
+    if ((int64_t)B * H > 65535) return fail(USV_ERR_UNSUPPORTED, "block_scores: B*H > 65535");
+    int rc;
+    if ((rc = check_view("q", q, sq, d)) != USV_OK) return rc;
+    if ((rc = check_view("k", k, sk, d)) != USV_OK) return rc;
+    if (scores == nullptr || ws == nullptr) return fail(USV_ERR_INVALID_ARG, "block_scores: null scores/ws");
+    if (!aligned16(scores) || !aligned16(ws))
+        return fail(USV_ERR_UNSUPPORTED, "block_scores: scores/ws not 16-byte aligned");
+    if (ws_bytes < usv_block_scores_workspace(B, H, Nq, Nk, d))
+        return fail(USV_ERR_WORKSPACE, "block_scores: workspace %zu < %zu", ws_bytes,
+                    usv_block_scores_workspace(B, H, Nq, Nk, d));
+    const int NBq = ceil_div(Nq, USV_BLOCK), NBk = ceil_div(Nk, USV_BLOCK);
+    float* qbar = static_cast<float*>(ws);
+    float* kbar = reinterpret_cast<float*>(static_cast<char*>(ws) +
+                                           align_up((size_t)B * H * NBq * d * sizeof(float), 256));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    PoolArgs a;
+    a.x[0] = static_cast<const __nv_bfloat16*>(q);
+    a.x[1] = static_cast<const __nv_bfloat16*>(k);
+    a.sb[0] = sq->sb; a.sh[0] = sq->sh; a.sn[0] = sq->sn;
+    a.sb[1] = sk->sb; a.sh[1] = sk->sh; a.sn[1] = sk->sn;
+    a.N[0] = Nq; a.N[1] = Nk; a.NB[0] = NBq; a.NB[1] = NBk;
+    a.out[0] = qbar; a.out[1] = kbar;
+    a.H = H;
+    dim3 pg(NBq > NBk ? NBq : NBk, B * H, 2);
+    if (d == 128) pool_kernel<128><<<pg, 128, 0, st>>>(a);
+    else pool_kernel<64><<<pg, 128, 0, st>>>(a);
+    USV_CHECK_LAUNCH("pool_kernel");
+
+    dim3 sg(ceil_div(NBk, 64), ceil_div(NBq, 64), B * H);
+    scores_kernel<<<sg, 256, 0, st>>>(qbar, kbar, scores, NBq, NBk, d, 1.0f / sqrtf((float)d));
+    USV_CHECK_LAUNCH("scores_kernel");
+    return USV_OK;
+}

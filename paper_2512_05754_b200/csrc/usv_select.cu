@@ -1,0 +1,144 @@
+// Top-k key-block selection: one CTA per score row.
+//
+// The row is mapped to order-preserving 32-bit keys in shared memory.  Four 8-bit radix passes
+// (most significant digit first) find the key T of the k-th largest element and the number of
+// elements strictly above it.  A final ordered pass emits, in ascending block index, every
+// index whose key is above T plus the first (k - above) indices whose key equals T, which is
+// exactly "k largest, ties to the lowest index".
+#include "usv_common.cuh"
+
+namespace usv {
+
+constexpr int SEL_THREADS = 256;
+constexpr int SEL_MAX_NB = 8192;
+
+struct SelHeads {
+    int k[USV_MAX_HEADS];
+};
+
+// Block-wide exclusive scan of one int per thread (SEL_THREADS threads); returns the exclusive
+// prefix and writes the block total to *total.  `scratch` holds >= 9 ints.
+__device__ __forceinline__ int block_excl_scan(int v, int* scratch, int* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int incl = warp_incl_scan(v);
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = lane < SEL_THREADS / 32 ? scratch[lane] : 0;
+        int wi = warp_incl_scan(w);
+        if (lane < SEL_THREADS / 32) scratch[lane] = wi - w;
+        if (lane == SEL_THREADS / 32 - 1) scratch[8] = wi;
+    }
+    __syncthreads();
+    const int res = scratch[warp] + incl - v;
+    *total = scratch[8];
+    __syncthreads();
+    return res;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* __restrict__ scores,
+                                                             int32_t* __restrict__ sel, int H,
+                                                             int NBq, int NBk, int kmax,
+                                                             const SelHeads heads) {
+    __shared__ uint32_t keys[SEL_MAX_NB];
+    __shared__ int hist[256];
+    __shared__ int scratch[9];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_remaining;
+
+    const int row = blockIdx.x;  // (b*H + h)*NBq + I
+    const int h = (row / NBq) % H;
+    const int k = heads.k[h];
+    const float* src = scores + (int64_t)row * NBk;
+    int32_t* out = sel + (int64_t)row * kmax;
+
+    for (int j = threadIdx.x; j < NBk; j += SEL_THREADS) keys[j] = float_key(src[j]);
+    if (threadIdx.x == 0) {
+        s_prefix = 0;
+        s_remaining = k;
+    }
+    __syncthreads();
+
+    // Radix select: after the pass for digit `shift`, s_prefix holds the top bits of T and
+    // s_remaining the rank of T among the elements that share those bits.
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        hist[threadIdx.x] = 0;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        const uint32_t mask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
+        for (int j = threadIdx.x; j < NBk; j += SEL_THREADS) {
+            const uint32_t key = keys[j];
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            // 256 bins, scanned from the top; each lane owns 8 consecutive bins.
+            const int lane = threadIdx.x;
+            const int remaining = s_remaining;  // read by every lane before the scan's shuffles
+            int local[8], sum = 0;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                local[t] = hist[255 - (lane * 8 + t)];
+                sum += local[t];
+            }
+            const int incl = warp_incl_scan(sum);
+            int before = incl - sum;  // elements in bins above this lane's bins
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                if (before < remaining && remaining <= before + local[t]) {
+                    s_prefix = prefix | ((uint32_t)(255 - (lane * 8 + t)) << shift);
+                    s_remaining = remaining - before;
+                }
+                before += local[t];
+            }
+        }
+        __syncthreads();
+    }
+    const uint32_t T = s_prefix;
+    const int need_eq = s_remaining;  // how many elements equal to T are kept (lowest indices)
+
+    int base_out = 0, base_eq = 0;
+    for (int j0 = 0; j0 < NBk; j0 += SEL_THREADS) {
+        const int j = j0 + threadIdx.x;
+        const uint32_t key = j < NBk ? keys[j] : 0u;
+        const int is_gt = (j < NBk && key > T) ? 1 : 0;
+        const int is_eq = (j < NBk && key == T) ? 1 : 0;
+        int tot_eq, tot_out;
+        const int eq_rank = base_eq + block_excl_scan(is_eq, scratch, &tot_eq);
+        const int take = is_gt | (is_eq && eq_rank < need_eq);
+        const int p = base_out + block_excl_scan(take, scratch, &tot_out);
+        if (take) out[p] = j;
+        base_eq += tot_eq;
+        base_out += tot_out;
+    }
+    for (int t = k + threadIdx.x; t < kmax; t += SEL_THREADS) out[t] = -1;
+}
+
+}  // namespace usv
+
+extern "C" int usv_select_blocks(int B, int H, int NBq, int NBk, const float* scores,
+                                 const int32_t* k_per_head, int kmax, int32_t* sel, void* stream) {
+    using namespace usv;
+    if (B <= 0 || H <= 0 || NBq <= 0 || NBk <= 0)
+        return fail(USV_ERR_INVALID_ARG, "select_blocks: B,H,NBq,NBk must be positive");
+    if (H > USV_MAX_HEADS) return fail(USV_ERR_UNSUPPORTED, "select_blocks: H > %d", USV_MAX_HEADS);
+    if (NBk > SEL_MAX_NB) return fail(USV_ERR_UNSUPPORTED, "select_blocks: NBk > %d", SEL_MAX_NB);
+    if (scores == nullptr || sel == nullptr || k_per_head == nullptr)
+        return fail(USV_ERR_INVALID_ARG, "select_blocks: null pointer");
+    SelHeads heads;
+    int kmx = 0;
+    for (int h = 0; h < H; ++h) {
+        if (k_per_head[h] < 1 || k_per_head[h] > NBk)
+            return fail(USV_ERR_INVALID_ARG, "select_blocks: k_per_head[%d]=%d outside [1,%d]", h,
+                        k_per_head[h], NBk);
+        heads.k[h] = k_per_head[h];
+        kmx = k_per_head[h] > kmx ? k_per_head[h] : kmx;
+    }
+    if (kmax < kmx) return fail(USV_ERR_INVALID_ARG, "select_blocks: kmax=%d < max k=%d", kmax, kmx);
+    const int64_t rows = (int64_t)B * H * NBq;
+    if (rows > 2147483647LL) return fail(USV_ERR_UNSUPPORTED, "select_blocks: too many rows");
+    select_kernel<<<(unsigned)rows, SEL_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+        scores, sel, H, NBq, NBk, kmax, heads);
+    USV_CHECK_LAUNCH("select_kernel");
+    return USV_OK;
+}
