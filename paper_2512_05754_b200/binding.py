@@ -139,7 +139,10 @@ def sparse_attn_fwd(q, k, v, sel, k_per_head, N=None, scale=0.0, out=None, retur
     kmax = sel.shape[3]
     karr, _ = _k_array(k_per_head, H)
     if out is None:
-        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=q.device)
+        if q.is_contiguous():
+            out = torch.empty_like(q)
+        else:   # token-major memory [B,N,H,d], returned as a [B,H,N,d] view
+            out = torch.empty((B, n, H, d), dtype=q.dtype, device=q.device).permute(0, 2, 1, 3)
     so = _view(out, "o")
     o32 = torch.empty((B, H, N, d), dtype=torch.float32, device=q.device) if return_f32 else None
     lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if return_lse else None

@@ -120,6 +120,10 @@ def check_merge_plan(plan_gpu, metric_cpu, grid, part, r, src_sample=None):
             ref_merged, _ = oracle.merge_select(idx, u[b], r)
             stats.setdefault("topr_differ", 0)
             stats["topr_differ"] += int((merged[idx] != ref_merged).sum())
+        # the selection step on its own: given the GPU's fp32 confidences, the merged set must be
+        # exactly the oracle's top-r of those same values (ties to the lowest source index)
+        ref_sel, _ = oracle.merge_select(src.astype(np.int32), gu[b, src].astype(np.float64), r)
+        assert np.array_equal(merged[src], ref_sel), "top-r of the GPU's own confidences"
     pos_ref, nm = oracle.merge_positions(dst_of, grid, part)
     assert nm == N - r and np.array_equal(pos, pos_ref), "pos must follow from dst_of exactly"
     return stats
