@@ -73,6 +73,34 @@ int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void* q, const u
                      size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * usv_block_scores for callers that cannot hand over scratch memory.  (The paper has no
+ * counterpart: this is a packaging variant of the entry point above, same arithmetic.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- inside a region that
+ * must not call cudaMalloc (an allocator-frozen section of a host framework, a plugin
+ * that is only given tensors, a real-time loop with a fixed memory budget) and that has no
+ * spare buffer to lend as `ws`.  Here the pooled block means live in a fixed array that is part
+ * of the library image: USV_NOALLOC_SCRATCH_BYTES of device memory are reserved on every GPU
+ * that loads the library, for as long as it stays loaded.
+ *
+ *   - Same arguments and results as usv_block_scores minus ws/ws_bytes.  Nothing is allocated
+ *     or freed, by the CUDA runtime or any other library.
+ *   - The request is rejected (USV_ERR_WORKSPACE, nothing launched) when
+ *     usv_block_scores_workspace(B,H,Nq,Nk,d) exceeds USV_NOALLOC_SCRATCH_BYTES.
+ *   - The first call on each device looks up the array's device address (a one-off, synchronous
+ *     runtime query with that device current).  Make that first call before starting any
+ *     stream capture on the device.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call left; every
+ *     element a call reads is first written by that same call, so nothing needs clearing.  Two
+ *     calls whose kernels overlap on the GPU (different streams, no ordering) race on it:
+ *     serialise them.
+ */
+#define USV_NOALLOC_SCRATCH_BYTES (8u << 20)
+int usv_block_scores_noalloc(int B, int H, int Nq, int Nk, int d, const void* q,
+                             const usv_strides* sq, const void* k, const usv_strides* sk,
+                             float* scores, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Top-k key-block selection (Fig. 2 caption, "top-k cube selection").  For each (b,h,I) the
  * k_per_head[h] key blocks with the largest score are kept; equal scores are resolved in favour
  * of the lower block index.  The kept indices are written in ascending order; the remainder of

@@ -5,6 +5,6 @@ marshalling only, every step of the path runs in the library's CUDA kernels.  Py
 device memory and streams.
 """
 from .binding import (  # noqa: F401
-    USVError, lib, lib_path, block_scores, select_blocks, sparse_attn_fwd, token_merge,
+    USVError, lib, lib_path, block_scores, block_scores_noalloc, select_blocks, sparse_attn_fwd, token_merge,
     token_unmerge, MergePlan, workspace_status, build_info, BLOCK,
 )

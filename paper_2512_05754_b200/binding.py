@@ -113,6 +113,26 @@ def block_scores(q, k, Nq=None, Nk=None, out=None):
     return out
 
 
+def block_scores_noalloc(q, k, Nq=None, Nk=None, out=None):
+    """block_scores for callers that must not allocate and have no scratch buffer to lend: the
+    pooled means go to a fixed array inside the library (8 MiB per GPU), so only shapes whose
+    scratch fits are accepted.  `out` should be passed by such callers (otherwise this wrapper
+    allocates the result tensor through torch, which the C entry point itself never does).
+    Calls on one device share the array: do not let two of them overlap on the GPU, and make the
+    first call on a device outside any stream capture."""
+    sq, sk = _view(q, "q"), _view(k, "k")
+    B, H, nq, d = q.shape
+    Nq = nq if Nq is None else int(Nq)
+    Nk = k.shape[2] if Nk is None else int(Nk)
+    NBq, NBk = (Nq + BLOCK - 1) // BLOCK, (Nk + BLOCK - 1) // BLOCK
+    if out is None:
+        out = torch.empty((B, H, NBq, NBk), dtype=torch.float32, device=q.device)
+    _check(lib().usv_block_scores_noalloc(B, H, Nq, Nk, d, _ptr(q), ctypes.byref(sq), _ptr(k),
+                                          ctypes.byref(sk), _ptr(out), _stream(q.device)),
+           "usv_block_scores_noalloc")
+    return out
+
+
 def select_blocks(scores, k_per_head, kmax=None, out=None):
     """Top-k key blocks per (b,h,I), ascending, ties to the lowest index; int32 [B,H,NBq,kmax]."""
     if scores.dtype != torch.float32 or not scores.is_cuda or not scores.is_contiguous():

@@ -173,3 +173,80 @@ extern "C" int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void*
     USV_CHECK_LAUNCH("scores_kernel");
     return USV_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Variant without caller scratch: the pooled means go to a fixed array inside the library image.
+// For callers that may neither allocate device memory nor lend a buffer (allocator-frozen
+// sections of a host framework, plugins that only receive tensors, fixed-budget loops).
+
+namespace usv {
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[USV_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static void* g_noalloc_ptr[kMaxDevices] = {};  // device address of the array, per device
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not an address a kernel
+// can use; the real per-device address has to be asked for once, with that device current.
+static int noalloc_scratch(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "block_scores_noalloc: cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices) return fail(USV_ERR_UNSUPPORTED, "block_scores_noalloc: device %d out of range", dev);
+    void* p = __atomic_load_n(&g_noalloc_ptr[dev], __ATOMIC_ACQUIRE);
+    if (p == nullptr) {
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess || p == nullptr)
+            return fail(USV_ERR_CUDA, "block_scores_noalloc: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        __atomic_store_n(&g_noalloc_ptr[dev], p, __ATOMIC_RELEASE);  // same value from any thread
+    }
+    *out = p;
+    return USV_OK;
+}
+
+}  // namespace usv
+
+extern "C" int usv_block_scores_noalloc(int B, int H, int Nq, int Nk, int d, const void* q,
+                                        const usv_strides* sq, const void* k,
+                                        const usv_strides* sk, float* scores, void* stream) {
+    using namespace usv;
+    if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0)
+        return fail(USV_ERR_INVALID_ARG, "block_scores_noalloc: B,H,Nq,Nk must be positive");
+    if (d != 64 && d != 128) return fail(USV_ERR_UNSUPPORTED, "block_scores_noalloc: d=%d (need 64 or 128)", d);
+    if ((int64_t)B * H > 65535) return fail(USV_ERR_UNSUPPORTED, "block_scores_noalloc: B*H > 65535");
+    int rc;
+    if ((rc = check_view("q", q, sq, d)) != USV_OK) return rc;
+    if ((rc = check_view("k", k, sk, d)) != USV_OK) return rc;
+    if (scores == nullptr) return fail(USV_ERR_INVALID_ARG, "block_scores_noalloc: null scores");
+    if (!aligned16(scores)) return fail(USV_ERR_UNSUPPORTED, "block_scores_noalloc: scores not 16-byte aligned");
+    const size_t need = usv_block_scores_workspace(B, H, Nq, Nk, d);
+    if (need > (size_t)USV_NOALLOC_SCRATCH_BYTES)
+        return fail(USV_ERR_WORKSPACE,
+                    "block_scores_noalloc: needs %zu bytes of scratch, the built-in array holds %u; "
+                    "use usv_block_scores with a caller workspace for this size",
+                    need, (unsigned)USV_NOALLOC_SCRATCH_BYTES);
+    void* scratch = nullptr;
+    if ((rc = noalloc_scratch(&scratch)) != USV_OK) return rc;
+
+    const int NBq = ceil_div(Nq, USV_BLOCK), NBk = ceil_div(Nk, USV_BLOCK);
+    float* qbar = static_cast<float*>(scratch);
+    float* kbar = reinterpret_cast<float*>(static_cast<char*>(scratch) +
+                                           align_up((size_t)B * H * NBq * d * sizeof(float), 256));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PoolArgs a;
+    a.x[0] = static_cast<const __nv_bfloat16*>(q);
+    a.x[1] = static_cast<const __nv_bfloat16*>(k);
+    a.sb[0] = sq->sb; a.sh[0] = sq->sh; a.sn[0] = sq->sn;
+    a.sb[1] = sk->sb; a.sh[1] = sk->sh; a.sn[1] = sk->sn;
+    a.N[0] = Nq; a.N[1] = Nk; a.NB[0] = NBq; a.NB[1] = NBk;
+    a.out[0] = qbar; a.out[1] = kbar;
+    a.H = H;
+    dim3 pg(NBq > NBk ? NBq : NBk, B * H, 2);
+    if (d == 128) pool_kernel<128><<<pg, 128, 0, st>>>(a);
+    else pool_kernel<64><<<pg, 128, 0, st>>>(a);
+    USV_CHECK_LAUNCH("pool_kernel (noalloc)");
+    dim3 sg(ceil_div(NBk, 64), ceil_div(NBq, 64), B * H);
+    scores_kernel<<<sg, 256, 0, st>>>(qbar, kbar, scores, NBq, NBk, d, 1.0f / sqrtf((float)d));
+    USV_CHECK_LAUNCH("scores_kernel (noalloc)");
+    return USV_OK;
+}

@@ -1,0 +1,54 @@
+"""The allocation-free variant of the block-score entry point.
+
+Some hosts of this library may not allocate device memory at the point where they call it and
+have no scratch buffer to pass (an allocator-frozen section of a framework, a plugin that only
+receives tensors).  usv_block_scores_noalloc serves them from a fixed array inside the library.
+It must give exactly what usv_block_scores gives, call after call, although every call reuses the
+same array and finds the previous call's contents in it.  Collected last on purpose."""
+import ctypes
+
+import pytest
+import torch
+
+import usv_inputs as ui
+
+
+def test_oversize_request_is_rejected_on_the_host():
+    from paper_2512_05754_b200 import binding
+    L = binding.lib()
+
+    class S(ctypes.Structure):
+        _fields_ = [("sb", ctypes.c_int64), ("sh", ctypes.c_int64), ("sn", ctypes.c_int64)]
+    p = ctypes.c_void_p(4096)             # never dereferenced: the size check comes first
+    N = 75600                             # 40 heads x 1182 blocks x 128 x 4 B x 2 = 48 MB > 8 MiB
+    s = S(40 * N * 128, N * 128, 128)
+    rc = L.usv_block_scores_noalloc(1, 40, N, N, 128, p, ctypes.byref(s), p, ctypes.byref(s), p, None)
+    assert rc == 3
+    assert b"built-in array" in L.usv_last_error()
+
+
+@pytest.mark.gpu
+def test_noalloc_matches_block_scores_on_two_calls_in_a_row():
+    import paper_2512_05754_b200 as usv
+    dev = torch.device("cuda", 0)
+    # first call: a shape that fills most of the array (12 heads x 400 blocks, d = 128)
+    wl = ui.Workload("noalloc_a", 200, 1, 12, 128, (16, 40, 40), (10,))
+    q, k, _ = ui.make_qkv(wl, device=dev)
+    N = wl.N - 13                                             # partial last block
+    out_a = torch.empty((1, 12, 400, 400), dtype=torch.float32, device=dev)
+    got_a = usv.block_scores_noalloc(q, k, N, N, out=out_a)
+    ref_a = usv.block_scores(q, k, N, N)
+    # second call right behind it: smaller, other head width, token-major layout; it finds the
+    # first call's pooled means still sitting in the shared array
+    wl2 = ui.Workload("noalloc_b", 201, 2, 3, 64, (5, 9, 11), (10,))
+    q2, k2, _ = ui.make_qkv(wl2, device=dev, layout="bnhd")
+    got_b = usv.block_scores_noalloc(q2, k2)
+    ref_b = usv.block_scores(q2, k2)
+    # and the first shape once more, to see that nothing of the second call leaks back
+    got_c = usv.block_scores_noalloc(q, k, N, N)
+    torch.cuda.synchronize()
+    tol = 2e-6 * max(1.0, ref_a.abs().max().item())
+    assert (got_a - ref_a).abs().max().item() <= tol
+    assert (got_b - ref_b).abs().max().item() <= 2e-6 * max(1.0, ref_b.abs().max().item())
+    assert (got_c - ref_a).abs().max().item() <= tol
+    assert got_a.data_ptr() == out_a.data_ptr()
