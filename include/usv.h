@@ -133,6 +133,11 @@ int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_str
                         int kmax, void* o, const usv_strides* so, float* o_f32, float* lse,
                         float scale, int impl, void* ws, size_t ws_bytes, void* stream);
 
+/* After usv_sparse_attn_fwd with impl 0: how many query blocks the tcgen05 kernel handed to the
+ * exact kernel because their softmax sums left the safe exponent range (normally 0).
+ * Synchronises `stream`.  ws is the workspace that call used. */
+int usv_sparse_attn_fallbacks(const void* ws, void* stream, int* count);
+
 /* Reads the device status word a kernel with bounded waits leaves in its workspace.
  * Synchronises `stream`.  Returns USV_OK, USV_ERR_TIMEOUT or USV_ERR_CUDA. */
 int usv_workspace_status(const void* ws, void* stream);

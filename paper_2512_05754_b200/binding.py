@@ -189,6 +189,16 @@ def workspace_status(device=None):
     return lib().usv_workspace_status(_ptr(ws), _stream(device))
 
 
+def sparse_attn_fallbacks(device=None):
+    """Query blocks of the last sparse_attn_fwd on this stream that were recomputed exactly."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    ws = _workspace(device, 256)
+    n = ctypes.c_int(0)
+    _check(lib().usv_sparse_attn_fallbacks(_ptr(ws), _stream(device), ctypes.byref(n)),
+           "usv_sparse_attn_fallbacks")
+    return n.value
+
+
 @dataclass
 class MergePlan:
     dst_of: torch.Tensor                 # int32 [B,N]

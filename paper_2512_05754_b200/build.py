@@ -52,7 +52,7 @@ def build(force=False, verbose=False):
             sys.stderr.write(out.decode())
         if p.returncode != 0:
             raise RuntimeError("nvcc failed on %s" % src)
-    subprocess.run([nvcc, "-shared", "-o", LIB] + objs + ["-lcuda"], check=True)
+    subprocess.run([nvcc, "-shared", "-o", LIB] + objs, check=True)
     return LIB
 
 

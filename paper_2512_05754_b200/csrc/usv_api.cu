@@ -57,3 +57,12 @@ extern "C" int usv_workspace_status(const void* ws, void* stream) {
         return usv::fail(USV_ERR_TIMEOUT, "device status word = 0x%x (a bounded wait gave up)", word);
     return USV_OK;
 }
+
+extern "C" int usv_sparse_attn_fallbacks(const void* ws, void* stream, int* count) {
+    if (ws == nullptr || count == nullptr) return usv::fail(USV_ERR_INVALID_ARG, "sparse_attn_fallbacks: null pointer");
+    cudaError_t e = cudaMemcpyAsync(count, static_cast<const char*>(ws) + 4, sizeof(int), cudaMemcpyDeviceToHost,
+                                    static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return usv::fail(USV_ERR_CUDA, "sparse_attn_fallbacks: %s", cudaGetErrorString(e));
+    return USV_OK;
+}

@@ -12,6 +12,12 @@ struct AttnArgs {
     float* o_f32;        // optional [B,H,N,D]
     float* lse;          // optional [B,H,N]
     unsigned int* status;  // optional device status word (bounded waits report here)
+    // Query blocks whose fixed-reference softmax left the safe range: the tcgen05 kernel appends
+    // their work ids here; the exact kernel, launched in list mode, recomputes them.
+    int* fallback_list;
+    int* fallback_count;
+    const int* work_list;   // list mode of the exact kernel (NULL = one CTA per query block)
+    const int* work_count;
     int B, H, N, NB, kmax;
     float scale_log2;    // softmax scale * log2(e)
     int k_per_head[USV_MAX_HEADS];
@@ -19,5 +25,7 @@ struct AttnArgs {
 };
 
 int launch_attn_mma(const AttnArgs& a, int d, cudaStream_t st);
+bool attn_tc_supported(const AttnArgs& a, int d);
+int launch_attn_tc(const AttnArgs& a, int d, cudaStream_t st);
 
 }  // namespace usv

@@ -4,8 +4,10 @@
 #include "usv_attn.cuh"
 
 extern "C" size_t usv_sparse_attn_workspace(int B, int H, int N, int d, int kmax) {
-    (void)B; (void)H; (void)N; (void)d; (void)kmax;
-    return 256;  // device status word (+ padding)
+    (void)d; (void)kmax;
+    if (B <= 0 || H <= 0 || N <= 0) return 0;
+    // status word + fallback counter (256-byte header), then the fallback work list
+    return 256 + usv::align_up((size_t)B * H * usv::ceil_div(N, USV_BLOCK) * sizeof(int), 256);
 }
 
 extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,
@@ -54,12 +56,23 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     a.o_f32 = o_f32;
     a.lse = lse;
     a.status = static_cast<unsigned int*>(ws);
+    a.fallback_count = reinterpret_cast<int*>(static_cast<char*>(ws) + 4);
+    a.fallback_list = reinterpret_cast<int*>(static_cast<char*>(ws) + 256);
+    a.work_list = nullptr;
+    a.work_count = nullptr;
     a.B = B; a.H = H; a.N = N; a.NB = NB; a.kmax = kmax;
     const float sc = scale == 0.f ? 1.0f / sqrtf((float)d) : scale;
     a.scale_log2 = sc * 1.4426950408889634f;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemsetAsync(ws, 0, 256, st);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: memset: %s", cudaGetErrorString(e));
-    (void)impl;
+    if (impl == 0 && attn_tc_supported(a, d)) {
+        int rc2 = launch_attn_tc(a, d, st);
+        if (rc2 != USV_OK) return rc2;
+        // exact recomputation of the (normally zero) query blocks the fast kernel reported
+        a.work_list = a.fallback_list;
+        a.work_count = a.fallback_count;
+        return launch_attn_mma(a, d, st);
+    }
     return launch_attn_mma(a, d, st);
 }

@@ -54,17 +54,15 @@ __device__ __forceinline__ void load_tile(__nv_bfloat16* dst, const __nv_bfloat1
 }
 
 template <int D>
-__global__ void __launch_bounds__(128) attn_mma_kernel(const AttnArgs a) {
+__device__ __forceinline__ void attn_mma_block(const AttnArgs& a, const int work, unsigned char* smem_raw) {
     constexpr int LD = MmaSmem<D>::LD;
     constexpr int TILE = MmaSmem<D>::TILE;
     constexpr int KT = D / 16;  // k-steps of QK^T
     constexpr int NT = D / 8;   // n-tiles of the output
-    extern __shared__ __align__(16) unsigned char smem_raw[];
     __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(smem_raw);
     __nv_bfloat16* Ks = Qs + TILE;
     __nv_bfloat16* Vs = Ks + 2 * TILE;
 
-    const int work = blockIdx.x;
     const int I = work % a.NB;
     const int bh_ord = work / a.NB;
     const int b = bh_ord / a.H;
@@ -268,9 +266,25 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const AttnArgs a) {
     }
 }
 
+// One CTA per query block, or (list mode) a fixed grid whose CTAs walk a device-side work list.
+template <int D>
+__global__ void __launch_bounds__(128) attn_mma_kernel(const AttnArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    if (a.work_list == nullptr) {
+        attn_mma_block<D>(a, blockIdx.x, smem_raw);
+        return;
+    }
+    const int n = *a.work_count;
+    for (int i = blockIdx.x; i < n; i += gridDim.x) {
+        attn_mma_block<D>(a, a.work_list[i], smem_raw);
+        __syncthreads();
+    }
+}
+
 int launch_attn_mma(const AttnArgs& a, int d, cudaStream_t st) {
-    const int64_t grid = (int64_t)a.B * a.H * a.NB;
+    int64_t grid = (int64_t)a.B * a.H * a.NB;
     if (grid > 2147483647LL) return fail(USV_ERR_UNSUPPORTED, "sparse_attn: too many query blocks");
+    if (a.work_list != nullptr && grid > 296) grid = 296;
     if (d == 128) {
         cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)MmaSmem<128>::BYTES);

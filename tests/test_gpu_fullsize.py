@@ -42,6 +42,7 @@ def _attention_parity(usv, q, k, v, N, kph, n_sample, seed, check_sel=True):
     o, o32 = usv.sparse_attn_fwd(q, k, v, sel, kph, N=N, return_f32=True)
     torch.cuda.synchronize()
     assert usv.workspace_status() == 0
+    print("query blocks recomputed by the exact kernel: %d" % usv.sparse_attn_fallbacks())
     qc, kc, vc = (t.cpu() for t in (q, k, v))
     sel_np = sel.cpu().numpy()
     if check_sel:
