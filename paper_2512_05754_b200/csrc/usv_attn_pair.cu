@@ -1,0 +1,431 @@
+// Block-sparse attention forward on the 5th-generation tensor cores (tcgen05 + TMEM + TMA).
+//
+// Formulation.  The selection is per 64-row query block, but the tensor-core datapath is 128 rows
+// high and a K/V tile costs as much shared-memory bandwidth to stage as to multiply.  One CTA
+// therefore owns TWO query blocks (rows 0-63 = block A, rows 64-127 = block B of one head) and
+// walks the ascending UNION of their two key-block lists, two key blocks (128 keys) per tile:
+//
+//     S[128 q x 128 keys]  = Q . K_tile^T      tcgen05.mma, A = Q resident in TMEM, B = K in smem
+//     O[128 q x 128 d]    += P . V_tile        tcgen05.mma, A = P (bf16) in TMEM,   B = V in smem
+//
+// A key block that only one of the two lists holds is masked for the other half of the rows
+// (its softmax weights are written as zero), so the result is exactly the per-block selection.
+// Neighbouring query blocks of video tokens select largely the same key blocks, which is what
+// makes the shared tile pay.
+//
+// Query rows live on TMEM lanes: softmax thread i owns row i, so maxima and sums need no
+// cross-thread traffic.  The softmax reference of a row (the value subtracted inside the
+// exponential) is fixed at the row maximum over the first key block the row may see and never
+// changes, so O needs no rescaling; the exponent range of fp32/bf16 absorbs later, larger
+// logits.  Rows whose sum leaves [2^-100, 2^100] are reported in a list and recomputed by the
+// exact online-softmax kernel, so the result never depends on that assumption.
+//
+// CTA = 6 warps: warps 0-3 softmax/epilogue (thread i <-> TMEM lane i), warp 4 TMA producer,
+// warp 5 MMA issuer and TMEM owner.  P overwrites the first half of the S buffer it came from.
+// All waits are bounded; a wait that gives up sets the device status word and every role leaves
+// its loop.
+#include "usv_attn.cuh"
+#include "usv_tcgen05.cuh"
+
+namespace usv {
+
+namespace pr {
+
+using namespace t5;
+
+constexpr int D = 128;
+constexpr int STAGES = 3;                       // K and V tile stages
+constexpr int MAX_NB = 4096;                    // key blocks per sequence this kernel covers
+constexpr uint32_t TILE_BYTES = 128 * D * 2;    // 32 KB: two 64-key blocks, [d-half][128 keys][128 B]
+constexpr uint32_t SM_K = 0;
+constexpr uint32_t SM_V = SM_K + STAGES * TILE_BYTES;
+constexpr uint32_t SM_BAR = SM_V + STAGES * TILE_BYTES;
+// barrier slots (8 bytes each)
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = B_KFULL + STAGES, B_VFULL = B_KEMPTY + STAGES,
+       B_VEMPTY = B_VFULL + STAGES, B_SFULL = B_VEMPTY + STAGES, B_PFULL = B_SFULL + 2,
+       B_OFULL = B_PFULL + 2, B_COUNT };
+static_assert(B_COUNT <= 32, "barrier area");
+constexpr uint32_t SM_MISC = SM_BAR + 8 * 32;            // tmem base, abort flag, flags, union size
+constexpr uint32_t SM_BITS = SM_MISC + 64;               // two bitmaps of MAX_NB bits
+constexpr uint32_t SM_LIST = SM_BITS + 2 * (MAX_NB / 8); // int[MAX_NB]: (key block << 2) | in-A | in-B << 1
+constexpr uint32_t SM_TOTAL = SM_LIST + MAX_NB * 4;
+constexpr size_t SMEM_BYTES = SM_TOTAL + 1024;           // + slack for 1024-byte alignment
+
+// TMEM columns: Q (bf16 pairs) | S/P buffer 0 | S/P buffer 1 | O
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t TQ = 0, TS = 64, TO = 320;
+
+__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+struct Maps {
+    CUtensorMap k, v;
+};
+
+// exp2 of 32 scaled logits -> 16 packed bf16 pairs; returns the sum of the ROUNDED weights
+template <bool MASKED>
+__device__ __forceinline__ float weights32(const uint32_t* sr, uint32_t* pk, float c, float nref, int col0,
+                                           int nvalid) {
+    float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float p0 = ex2(fmaf(__uint_as_float(sr[2 * j]), c, nref));
+        float p1 = ex2(fmaf(__uint_as_float(sr[2 * j + 1]), c, nref));
+        if (MASKED) {
+            if (col0 + 2 * j >= nvalid) p0 = 0.f;
+            if (col0 + 2 * j + 1 >= nvalid) p1 = 0.f;
+        }
+        const uint32_t w = pack_bf16x2(p0, p1);
+        acc0 += __uint_as_float(w << 16);
+        acc1 += __uint_as_float(w & 0xffff0000u);
+        pk[j] = w;
+    }
+    return acc0 + acc1;
+}
+
+__global__ void __launch_bounds__(192, 1)
+attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* sm = smem_raw + (base - raw);
+    auto bar = [&](int i) { return base + SM_BAR + 8u * i; };
+    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(sm + SM_MISC);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(sm + SM_MISC + 4);
+    volatile int* s_flag = reinterpret_cast<volatile int*>(sm + SM_MISC + 8);   // [2]
+    volatile int* s_nu = reinterpret_cast<volatile int*>(sm + SM_MISC + 16);
+    uint32_t* s_bits = reinterpret_cast<uint32_t*>(sm + SM_BITS);
+    int* s_list = reinterpret_cast<int*>(sm + SM_LIST);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int NB = a.NB, N = a.N;
+    const int NP = (NB + 1) >> 1;                 // query-block pairs per (b, h)
+    const int pair = blockIdx.x % NP;
+    const int bh_ord = blockIdx.x / NP;
+    const int b = bh_ord / a.H;
+    const int h = a.head_order[bh_ord % a.H];
+    const int kh = a.k_per_head[h];
+    const int IA = 2 * pair;
+    const int IB = (2 * pair + 1 < NB) ? 2 * pair + 1 : -1;
+    const int nwords = (NB + 31) >> 5;
+
+    // ---- set-up: barriers, TMEM, ascending union of the two selection rows
+    if (threadIdx.x == 0) {
+        mbar_init(bar(B_QFULL), 128);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar(B_KFULL + s), 1);
+            mbar_init(bar(B_KEMPTY + s), 1);
+            mbar_init(bar(B_VFULL + s), 1);
+            mbar_init(bar(B_VEMPTY + s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(B_SFULL + s), 1);
+            mbar_init(bar(B_PFULL + s), 128);
+        }
+        mbar_init(bar(B_OFULL), 1);
+        *s_abort = 0;
+        s_flag[0] = 0;
+        s_flag[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(base + SM_MISC), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (warp < 4) {
+        const int tid = threadIdx.x;
+        uint32_t* bitsA = s_bits;
+        uint32_t* bitsB = s_bits + MAX_NB / 32;
+        for (int w = tid; w < nwords; w += 128) {
+            bitsA[w] = 0;
+            bitsB[w] = 0;
+        }
+        softmax_bar();
+        const int32_t* selA = a.sel + (((int64_t)b * a.H + h) * NB + IA) * a.kmax;
+        for (int t = tid; t < kh; t += 128) {
+            const int J = selA[t];
+            if (J >= 0 && J < NB) atomicOr(&bitsA[J >> 5], 1u << (J & 31));
+        }
+        if (IB >= 0) {
+            const int32_t* selB = selA + a.kmax;
+            for (int t = tid; t < kh; t += 128) {
+                const int J = selB[t];
+                if (J >= 0 && J < NB) atomicOr(&bitsB[J >> 5], 1u << (J & 31));
+            }
+        }
+        softmax_bar();
+        if (warp == 0) {
+            int running = 0;
+            for (int w0 = 0; w0 < nwords; w0 += 32) {
+                const int w = w0 + lane;
+                const uint32_t ba = w < nwords ? bitsA[w] : 0u;
+                const uint32_t bb = w < nwords ? bitsB[w] : 0u;
+                uint32_t u = ba | bb;
+                const int incl = warp_incl_scan(__popc(u));
+                int off = running + incl - __popc(u);
+                while (u) {
+                    const int bit = __ffs(u) - 1;
+                    u &= u - 1;
+                    s_list[off++] = ((w * 32 + bit) << 2) | ((ba >> bit) & 1u) | (((bb >> bit) & 1u) << 1);
+                }
+                running += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (lane == 0) *s_nu = running;
+        }
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = *s_tmem;
+    const int nU = *s_nu;
+    const int T = (nU + 1) >> 1;   // 128-key tiles
+
+    if (warp == 4) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            for (int t = 0; t < T; ++t) {
+                const int s = t % STAGES;
+                const uint32_t ph = (t / STAGES) & 1;
+                const int J0 = s_list[2 * t] >> 2;
+                const int J1 = (2 * t + 1 < nU) ? (s_list[2 * t + 1] >> 2) : J0;  // odd tail: finite filler, masked
+                if (!mbar_wait(bar(B_KEMPTY + s), ph ^ 1, s_abort, a.status, 0x1)) break;
+                mbar_expect_tx(bar(B_KFULL + s), TILE_BYTES);
+                const uint32_t kd = base + SM_K + s * TILE_BYTES;
+                tma_load_4d(kd, &maps.k, bar(B_KFULL + s), 0, J0 * USV_BLOCK, h, b);
+                tma_load_4d(kd + 8192, &maps.k, bar(B_KFULL + s), 0, J1 * USV_BLOCK, h, b);
+                tma_load_4d(kd + 16384, &maps.k, bar(B_KFULL + s), 64, J0 * USV_BLOCK, h, b);
+                tma_load_4d(kd + 24576, &maps.k, bar(B_KFULL + s), 64, J1 * USV_BLOCK, h, b);
+                if (!mbar_wait(bar(B_VEMPTY + s), ph ^ 1, s_abort, a.status, 0x2)) break;
+                mbar_expect_tx(bar(B_VFULL + s), TILE_BYTES);
+                const uint32_t vd = base + SM_V + s * TILE_BYTES;
+                tma_load_4d(vd, &maps.v, bar(B_VFULL + s), 0, J0 * USV_BLOCK, h, b);
+                tma_load_4d(vd + 8192, &maps.v, bar(B_VFULL + s), 0, J1 * USV_BLOCK, h, b);
+                tma_load_4d(vd + 16384, &maps.v, bar(B_VFULL + s), 64, J0 * USV_BLOCK, h, b);
+                tma_load_4d(vd + 24576, &maps.v, bar(B_VFULL + s), 64, J1 * USV_BLOCK, h, b);
+            }
+        }
+    } else if (warp == 5) {
+        // ================= MMA issuer =================
+        if (lane == 0 && T > 0) {
+            constexpr uint32_t IDESC_S = instr_desc(128, 128, 0, 0);   // Q (TMEM) x K (K-major)
+            constexpr uint32_t IDESC_O = instr_desc(128, 128, 0, 1);   // P (TMEM) x V (MN-major)
+            bool ok = mbar_wait(bar(B_QFULL), 0, s_abort, a.status, 0x4);
+            auto issue_s = [&](int t) -> bool {
+                const int s = t % STAGES;
+                const uint32_t ph = (t / STAGES) & 1;
+                const int sb = t & 1;
+                if (!mbar_wait(bar(B_KFULL + s), ph, s_abort, a.status, 0x8)) return false;
+                fence_after();
+                const uint32_t kd = base + SM_K + s * TILE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+                    umma_ts(tmem + TS + sb * 128, tmem + TQ + ks * 8, smem_desc(kd + off, 16, 1024), IDESC_S,
+                            ks > 0);
+                }
+                umma_commit(bar(B_KEMPTY + s));
+                umma_commit(bar(B_SFULL + sb));
+                return true;
+            };
+            if (ok) ok = issue_s(0);
+            for (int t = 0; ok && t < T; ++t) {
+                // S of the next tile goes to the other buffer; the MMA before it that read P from
+                // there (tile t-1) was issued earlier by this thread, and MMAs execute in order.
+                if (t + 1 < T) {
+                    ok = issue_s(t + 1);
+                    if (!ok) break;
+                }
+                const int s = t % STAGES;
+                const uint32_t ph = (t / STAGES) & 1;
+                const int sb = t & 1;
+                if (!mbar_wait(bar(B_VFULL + s), ph, s_abort, a.status, 0x20)) break;
+                if (!mbar_wait(bar(B_PFULL + sb), (t >> 1) & 1, s_abort, a.status, 0x40)) break;
+                fence_after();
+                const uint32_t vd = base + SM_V + s * TILE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    umma_ts(tmem + TO, tmem + TS + sb * 128 + ks * 8, smem_desc(vd + ks * 2048, 16384, 1024),
+                            IDESC_O, (t > 0 || ks > 0));
+                }
+                umma_commit(bar(B_VEMPTY + s));
+                if (t == T - 1) umma_commit(bar(B_OFULL));
+            }
+        }
+    } else if (T > 0) {
+        // ================= softmax + epilogue (thread i <-> TMEM lane i <-> query row) ==========
+        const int tid = threadIdx.x;
+        const int side = tid >> 6;                       // 0: block A, 1: block B (uniform per warp)
+        const int Iq = side ? IB : IA;
+        const int row = Iq * USV_BLOCK + (tid & 63);
+        const bool live = Iq >= 0 && row < N;
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        const float c = a.scale_log2;
+        {
+            // this thread's query row -> TMEM (two bf16 of consecutive d per 32-bit column)
+            const uint4* src = reinterpret_cast<const uint4*>(a.q + b * a.sq.sb + h * a.sq.sh + (int64_t)row * a.sq.sn);
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                uint32_t r[16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 v = live ? __ldg(src + c4 * 4 + i) : make_uint4(0, 0, 0, 0);
+                    r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+                }
+                tmem_st16(lane_base + TQ + c4 * 16, r);
+            }
+            tmem_wait_st();
+            fence_before();
+            mbar_arrive(bar(B_QFULL));
+        }
+        float nref = 0.f;         // minus the softmax reference (base-2, scaled)
+        bool have_ref = false;
+        float lr = 0.f;           // sum of the rounded weights of this row
+        bool ok = true;
+        for (int t = 0; t < T; ++t) {
+            const int sb = t & 1;
+            if (!mbar_wait(bar(B_SFULL + sb), (t >> 1) & 1, s_abort, a.status, 0x80)) { ok = false; break; }
+            fence_after();
+            const uint32_t sbase = lane_base + TS + sb * 128;
+#pragma unroll
+            for (int hb = 0; hb < 2; ++hb) {
+                const int slot = 2 * t + hb;
+                const int e = slot < nU ? s_list[slot] : 0;
+                const bool mine = (e >> side) & 1;
+                if (mine) {
+                    const int nvalid = N - (e >> 2) * USV_BLOCK;   // keys of this block with index < N
+                    uint32_t s0[32], s1[32];
+                    tmem_ld32(sbase + hb * 64, s0);
+                    tmem_ld32(sbase + hb * 64 + 32, s1);
+                    tmem_wait_ld();
+                    if (!have_ref) {
+                        float mx = -INFINITY;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < nvalid) mx = fmaxf(mx, __uint_as_float(s0[j]));
+                            if (j + 32 < nvalid) mx = fmaxf(mx, __uint_as_float(s1[j]));
+                        }
+                        nref = -mx * c;
+                        have_ref = true;
+                    }
+                    uint32_t pk[16];
+                    if (nvalid >= USV_BLOCK) {
+                        lr += weights32<false>(s0, pk, c, nref, 0, nvalid);
+                        tmem_st16(sbase + hb * 32, pk);
+                        lr += weights32<false>(s1, pk, c, nref, 32, nvalid);
+                        tmem_st16(sbase + hb * 32 + 16, pk);
+                    } else {
+                        lr += weights32<true>(s0, pk, c, nref, 0, nvalid);
+                        tmem_st16(sbase + hb * 32, pk);
+                        lr += weights32<true>(s1, pk, c, nref, 32, nvalid);
+                        tmem_st16(sbase + hb * 32 + 16, pk);
+                    }
+                } else {
+                    uint32_t z[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) z[j] = 0u;
+                    tmem_st16(sbase + hb * 32, z);
+                    tmem_st16(sbase + hb * 32 + 16, z);
+                }
+            }
+            tmem_wait_st();
+            fence_before();
+            mbar_arrive(bar(B_PFULL + sb));
+        }
+        // ---- epilogue
+        if (ok) ok = mbar_wait(bar(B_OFULL), 0, s_abort, a.status, 0x200);
+        if (ok) {
+            fence_after();
+            const bool in_range = lr > 7.9e-31f && lr < 1.2e30f;   // ~[2^-100, 2^100]
+            if (live && !in_range) s_flag[side] = 1;
+            const float inv = lr > 0.f ? 1.0f / lr : 0.f;
+            if (a.lse != nullptr && live)
+                a.lse[((int64_t)b * a.H + h) * N + row] = (log2f(lr) - nref) * 0.69314718055994531f;
+            float* o32 = (a.o_f32 != nullptr && live) ? a.o_f32 + (((int64_t)b * a.H + h) * N + row) * D : nullptr;
+            unsigned char* stage = sm + SM_K;   // [128 rows][256 B], 16-byte chunks XOR-swizzled by row
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t orr[32];
+                tmem_ld32(lane_base + TO + ch * 32, orr);
+                tmem_wait_ld();
+                float f[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(orr[j]) * inv;
+                if (o32 != nullptr) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<float4*>(o32 + ch * 32 + j * 4) =
+                            make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int cc = ch * 4 + i;
+                    *reinterpret_cast<uint4*>(stage + tid * 256 + ((cc ^ (tid & 15)) << 4)) = float8_to_bf16x8(f + 8 * i);
+                }
+            }
+            softmax_bar();
+            __nv_bfloat16* O = a.o + b * a.so.sb + h * a.so.sh;
+#pragma unroll 4
+            for (int idx = tid; idx < 128 * 16; idx += 128) {
+                const int r = idx >> 4, cc = idx & 15;
+                const int Ir = r < 64 ? IA : IB;
+                const int grow = Ir * USV_BLOCK + (r & 63);
+                if (Ir >= 0 && grow < N)
+                    *reinterpret_cast<uint4*>(O + (int64_t)grow * a.so.sn + cc * 8) =
+                        *reinterpret_cast<const uint4*>(stage + r * 256 + ((cc ^ (r & 15)) << 4));
+            }
+        }
+    }
+
+    // ---- teardown
+    fence_before();
+    __syncthreads();
+    if (*s_abort) {
+        // give copies and MMAs that may still be in flight time to land before the CTA's
+        // shared memory and TMEM are handed back
+        const unsigned long long t0 = gtime();
+        while (gtime() - t0 < 2000000ull) { }
+        __syncthreads();
+    }
+    if (threadIdx.x < 2 && T > 0 && s_flag[threadIdx.x] && a.fallback_list != nullptr) {
+        const int slot = atomicAdd(a.fallback_count, 1);
+        a.fallback_list[slot] = bh_ord * NB + (threadIdx.x ? IB : IA);
+    }
+    if (T == 0) {
+        // no valid key block at all: defined output (zeros), as the exact kernel does
+        __nv_bfloat16* O = a.o + b * a.so.sb + h * a.so.sh;
+        for (int idx = threadIdx.x; idx < 128 * (D / 8); idx += blockDim.x) {
+            const int r = idx / (D / 8);
+            const int Ir = r < 64 ? IA : IB;
+            const int grow = Ir * USV_BLOCK + (r & 63);
+            if (Ir >= 0 && grow < N)
+                *reinterpret_cast<uint4*>(O + (int64_t)grow * a.so.sn + (idx % (D / 8)) * 8) = make_uint4(0, 0, 0, 0);
+        }
+    }
+    if (warp == 5) {
+        fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace pr
+
+bool attn_pair_supported(const AttnArgs& a, int d) {
+    return d == pr::D && a.NB <= pr::MAX_NB;
+}
+
+int launch_attn_pair(const AttnArgs& a, int d, cudaStream_t st) {
+    pr::Maps maps;
+    int rc;
+    if ((rc = t5::make_bhnd_map(&maps.k, a.k, a.sk, a.B, a.H, a.N, d, "k")) != USV_OK) return rc;
+    if ((rc = t5::make_bhnd_map(&maps.v, a.v, a.sv, a.B, a.H, a.N, d, "v")) != USV_OK) return rc;
+    const int64_t grid = (int64_t)a.B * a.H * ((a.NB + 1) / 2);
+    if (grid > 2147483647LL) return fail(USV_ERR_UNSUPPORTED, "sparse_attn: too many query blocks");
+    cudaError_t e = cudaFuncSetAttribute(pr::attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)pr::SMEM_BYTES);
+    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: smem attribute: %s", cudaGetErrorString(e));
+    pr::attn_pair_kernel<<<(unsigned)grid, 192, pr::SMEM_BYTES, st>>>(a, maps);
+    USV_CHECK_LAUNCH("attn_pair_kernel");
+    return USV_OK;
+}
+
+}  // namespace usv
