@@ -20,8 +20,10 @@
 // logits.  Rows whose sum leaves [2^-100, 2^100] are reported in a list and recomputed by the
 // exact online-softmax kernel, so the result never depends on that assumption.
 //
-// CTA = 6 warps: warps 0-3 softmax/epilogue (thread i <-> TMEM lane i), warp 4 TMA producer,
-// warp 5 MMA issuer and TMEM owner.  P overwrites the first half of the S buffer it came from.
+// CTA = 10 warps: warps 0-7 softmax/epilogue as two warpgroups that share the rows (thread i of
+// either group <-> TMEM lane i) and alternate tiles (group g: tiles t = g mod 2, S/P buffer g),
+// so that the load-exponentiate-store chains of two tiles overlap; warp 8 TMA producer, warp 9
+// MMA issuer and TMEM owner.  P overwrites part of the S buffer it came from.
 // All waits are bounded; a wait that gives up sets the device status word and every role leaves
 // its loop.
 #include "usv_attn.cuh"
@@ -43,19 +45,23 @@ constexpr uint32_t SM_BAR = SM_V + STAGES * TILE_BYTES;
 // barrier slots (8 bytes each)
 enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = B_KFULL + STAGES, B_VFULL = B_KEMPTY + STAGES,
        B_VEMPTY = B_VFULL + STAGES, B_SFULL = B_VEMPTY + STAGES, B_PFULL = B_SFULL + 2,
-       B_OFULL = B_PFULL + 2, B_COUNT };
+       B_OFULL = B_PFULL + 2, B_REF, B_EPI = B_REF + 2, B_COUNT = B_EPI + 2 };
 static_assert(B_COUNT <= 32, "barrier area");
 constexpr uint32_t SM_MISC = SM_BAR + 8 * 32;            // tmem base, abort flag, flags, union size
 constexpr uint32_t SM_BITS = SM_MISC + 64;               // two bitmaps of MAX_NB bits
 constexpr uint32_t SM_LIST = SM_BITS + 2 * (MAX_NB / 8); // int[MAX_NB]: (key block << 2) | in-A | in-B << 1
-constexpr uint32_t SM_TOTAL = SM_LIST + MAX_NB * 4;
+constexpr uint32_t SM_MAX = SM_LIST + MAX_NB * 4;        // float[128 rows] minus the softmax reference (+ spare)
+constexpr uint32_t SM_SUM = SM_MAX + 2 * 128 * 4;        // float[2 groups][128 rows] row sums
+constexpr uint32_t SM_TOTAL = SM_SUM + 2 * 128 * 4;
 constexpr size_t SMEM_BYTES = SM_TOTAL + 1024;           // + slack for 1024-byte alignment
 
 // TMEM columns: Q (bf16 pairs) | S/P buffer 0 | S/P buffer 1 | O
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TQ = 0, TS = 64, TO = 320;
 
-__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+constexpr int NSOFT = 256;   // softmax threads
+constexpr int NTHREADS = NSOFT + 64;
+__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 struct Maps {
     CUtensorMap k, v;
@@ -82,7 +88,7 @@ __device__ __forceinline__ float weights32(const uint32_t* sr, uint32_t* pk, flo
     return acc0 + acc1;
 }
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(NTHREADS, 1)
 attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -95,6 +101,8 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     volatile int* s_nu = reinterpret_cast<volatile int*>(sm + SM_MISC + 16);
     uint32_t* s_bits = reinterpret_cast<uint32_t*>(sm + SM_BITS);
     int* s_list = reinterpret_cast<int*>(sm + SM_LIST);
+    float* s_max = reinterpret_cast<float*>(sm + SM_MAX);
+    float* s_sum = reinterpret_cast<float*>(sm + SM_SUM);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NB = a.NB, N = a.N;
@@ -107,10 +115,11 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const int IA = 2 * pair;
     const int IB = (2 * pair + 1 < NB) ? 2 * pair + 1 : -1;
     const int nwords = (NB + 31) >> 5;
+    constexpr int W_TMA = NSOFT / 32, W_MMA = NSOFT / 32 + 1;
 
     // ---- set-up: barriers, TMEM, ascending union of the two selection rows
     if (threadIdx.x == 0) {
-        mbar_init(bar(B_QFULL), 128);
+        mbar_init(bar(B_QFULL), NSOFT / 32);       // one arrival per softmax warp
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar(B_KFULL + s), 1);
             mbar_init(bar(B_KEMPTY + s), 1);
@@ -119,36 +128,42 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(B_SFULL + s), 1);
-            mbar_init(bar(B_PFULL + s), 128);
+            mbar_init(bar(B_PFULL + s), 4);         // one arrival per warp of the group
         }
         mbar_init(bar(B_OFULL), 1);
+        // rendezvous of the softmax threads after the first bounded wait: mbarriers, so that they
+        // too can give up (a bar.sync would hang if one thread had left its loop)
+        mbar_init(bar(B_REF), 64);
+        mbar_init(bar(B_REF + 1), 64);
+        mbar_init(bar(B_EPI), NSOFT);
+        mbar_init(bar(B_EPI + 1), NSOFT);
         *s_abort = 0;
         s_flag[0] = 0;
         s_flag[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == W_MMA) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(base + SM_MISC), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (warp < 4) {
+    if (warp < W_TMA) {
         const int tid = threadIdx.x;
         uint32_t* bitsA = s_bits;
         uint32_t* bitsB = s_bits + MAX_NB / 32;
-        for (int w = tid; w < nwords; w += 128) {
+        for (int w = tid; w < nwords; w += NSOFT) {
             bitsA[w] = 0;
             bitsB[w] = 0;
         }
         softmax_bar();
         const int32_t* selA = a.sel + (((int64_t)b * a.H + h) * NB + IA) * a.kmax;
-        for (int t = tid; t < kh; t += 128) {
+        for (int t = tid; t < kh; t += NSOFT) {
             const int J = selA[t];
             if (J >= 0 && J < NB) atomicOr(&bitsA[J >> 5], 1u << (J & 31));
         }
         if (IB >= 0) {
             const int32_t* selB = selA + a.kmax;
-            for (int t = tid; t < kh; t += 128) {
+            for (int t = tid; t < kh; t += NSOFT) {
                 const int J = selB[t];
                 if (J >= 0 && J < NB) atomicOr(&bitsB[J >> 5], 1u << (J & 31));
             }
@@ -180,35 +195,41 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const int nU = *s_nu;
     const int T = (nU + 1) >> 1;   // 128-key tiles
 
-    if (warp == 4) {
-        // ================= TMA producer =================
-        if (lane == 0) {
-            for (int t = 0; t < T; ++t) {
-                const int s = t % STAGES;
-                const uint32_t ph = (t / STAGES) & 1;
-                const int J0 = s_list[2 * t] >> 2;
-                const int J1 = (2 * t + 1 < nU) ? (s_list[2 * t + 1] >> 2) : J0;  // odd tail: finite filler, masked
-                if (!mbar_wait(bar(B_KEMPTY + s), ph ^ 1, s_abort, a.status, 0x1)) break;
+    if (warp == W_TMA) {
+        // ================= TMA producer (whole warp in the loop, one elected lane issues) ======
+        for (int t = 0; t < T; ++t) {
+            const int s = t % STAGES;
+            const uint32_t ph = (t / STAGES) & 1;
+            const int J0 = s_list[2 * t] >> 2;
+            const int J1 = (2 * t + 1 < nU) ? (s_list[2 * t + 1] >> 2) : J0;  // odd tail: finite filler, masked
+            if (!mbar_wait(bar(B_KEMPTY + s), ph ^ 1, s_abort, a.status, 0x1)) break;
+            const uint32_t kd = base + SM_K + s * TILE_BYTES;
+            if (elect_one()) {
                 mbar_expect_tx(bar(B_KFULL + s), TILE_BYTES);
-                const uint32_t kd = base + SM_K + s * TILE_BYTES;
                 tma_load_4d(kd, &maps.k, bar(B_KFULL + s), 0, J0 * USV_BLOCK, h, b);
                 tma_load_4d(kd + 8192, &maps.k, bar(B_KFULL + s), 0, J1 * USV_BLOCK, h, b);
                 tma_load_4d(kd + 16384, &maps.k, bar(B_KFULL + s), 64, J0 * USV_BLOCK, h, b);
                 tma_load_4d(kd + 24576, &maps.k, bar(B_KFULL + s), 64, J1 * USV_BLOCK, h, b);
-                if (!mbar_wait(bar(B_VEMPTY + s), ph ^ 1, s_abort, a.status, 0x2)) break;
+            }
+            __syncwarp();
+            if (!mbar_wait(bar(B_VEMPTY + s), ph ^ 1, s_abort, a.status, 0x2)) break;
+            const uint32_t vd = base + SM_V + s * TILE_BYTES;
+            if (elect_one()) {
                 mbar_expect_tx(bar(B_VFULL + s), TILE_BYTES);
-                const uint32_t vd = base + SM_V + s * TILE_BYTES;
                 tma_load_4d(vd, &maps.v, bar(B_VFULL + s), 0, J0 * USV_BLOCK, h, b);
                 tma_load_4d(vd + 8192, &maps.v, bar(B_VFULL + s), 0, J1 * USV_BLOCK, h, b);
                 tma_load_4d(vd + 16384, &maps.v, bar(B_VFULL + s), 64, J0 * USV_BLOCK, h, b);
                 tma_load_4d(vd + 24576, &maps.v, bar(B_VFULL + s), 64, J1 * USV_BLOCK, h, b);
             }
+            __syncwarp();
         }
-    } else if (warp == 5) {
-        // ================= MMA issuer =================
-        if (lane == 0 && T > 0) {
+    } else if (warp == W_MMA) {
+        // ================= MMA issuer (whole warp in the loop, one elected lane issues) ========
+        if (T > 0) {
             constexpr uint32_t IDESC_S = instr_desc(128, 128, 0, 0);   // Q (TMEM) x K (K-major)
             constexpr uint32_t IDESC_O = instr_desc(128, 128, 0, 1);   // P (TMEM) x V (MN-major)
+            const uint64_t kdesc0 = smem_desc(base + SM_K, 16, 1024);       // + byte offset >> 4
+            const uint64_t vdesc0 = smem_desc(base + SM_V, 16384, 1024);
             bool ok = mbar_wait(bar(B_QFULL), 0, s_abort, a.status, 0x4);
             auto issue_s = [&](int t) -> bool {
                 const int s = t % STAGES;
@@ -216,21 +237,23 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 const int sb = t & 1;
                 if (!mbar_wait(bar(B_KFULL + s), ph, s_abort, a.status, 0x8)) return false;
                 fence_after();
-                const uint32_t kd = base + SM_K + s * TILE_BYTES;
+                const uint64_t kdesc = kdesc0 + ((s * TILE_BYTES) >> 4);
+                const uint32_t d_s = tmem + TS + sb * 128;
+                if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
-                    umma_ts(tmem + TS + sb * 128, tmem + TQ + ks * 8, smem_desc(kd + off, 16, 1024), IDESC_S,
-                            ks > 0);
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        umma_ts(d_s, tmem + TQ + ks * 8, kdesc + (((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
+                                IDESC_S, ks > 0);
+                    umma_commit(bar(B_KEMPTY + s));
+                    umma_commit(bar(B_SFULL + sb));
                 }
-                umma_commit(bar(B_KEMPTY + s));
-                umma_commit(bar(B_SFULL + sb));
+                __syncwarp();
                 return true;
             };
             if (ok) ok = issue_s(0);
             for (int t = 0; ok && t < T; ++t) {
                 // S of the next tile goes to the other buffer; the MMA before it that read P from
-                // there (tile t-1) was issued earlier by this thread, and MMAs execute in order.
+                // there (tile t-1) was issued earlier by the same lane, and MMAs execute in order.
                 if (t + 1 < T) {
                     ok = issue_s(t + 1);
                     if (!ok) break;
@@ -241,111 +264,163 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 if (!mbar_wait(bar(B_VFULL + s), ph, s_abort, a.status, 0x20)) break;
                 if (!mbar_wait(bar(B_PFULL + sb), (t >> 1) & 1, s_abort, a.status, 0x40)) break;
                 fence_after();
-                const uint32_t vd = base + SM_V + s * TILE_BYTES;
+                const uint64_t vdesc = vdesc0 + ((s * TILE_BYTES) >> 4);
+                const uint32_t a_p = tmem + TS + sb * 128;
+                if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    umma_ts(tmem + TO, tmem + TS + sb * 128 + ks * 8, smem_desc(vd + ks * 2048, 16384, 1024),
-                            IDESC_O, (t > 0 || ks > 0));
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_ts(tmem + TO, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vdesc + ((ks * 2048) >> 4),
+                                IDESC_O, (t > 0 || ks > 0));
+                    umma_commit(bar(B_VEMPTY + s));
+                    if (t == T - 1) umma_commit(bar(B_OFULL));
                 }
-                umma_commit(bar(B_VEMPTY + s));
-                if (t == T - 1) umma_commit(bar(B_OFULL));
+                __syncwarp();
             }
         }
     } else if (T > 0) {
-        // ================= softmax + epilogue (thread i <-> TMEM lane i <-> query row) ==========
-        const int tid = threadIdx.x;
-        const int side = tid >> 6;                       // 0: block A, 1: block B (uniform per warp)
+        // ===== softmax + epilogue: thread r of either group <-> TMEM lane r <-> query row r =====
+        const int grp = warp >> 2;                       // key block of each tile this group handles
+        const int r = threadIdx.x & 127;
+        const int side = r >> 6;                         // 0: block A, 1: block B (uniform per warp)
         const int Iq = side ? IB : IA;
-        const int row = Iq * USV_BLOCK + (tid & 63);
+        const int row = Iq * USV_BLOCK + (r & 63);
         const bool live = Iq >= 0 && row < N;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         const float c = a.scale_log2;
         {
-            // this thread's query row -> TMEM (two bf16 of consecutive d per 32-bit column)
-            const uint4* src = reinterpret_cast<const uint4*>(a.q + b * a.sq.sb + h * a.sq.sh + (int64_t)row * a.sq.sn);
+            // this thread's half of its query row -> TMEM (two bf16 of consecutive d per column)
+            const uint4* src = reinterpret_cast<const uint4*>(a.q + b * a.sq.sb + h * a.sq.sh +
+                                                              (int64_t)row * a.sq.sn + grp * 64);
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint32_t r[16];
+            for (int c4 = 0; c4 < 2; ++c4) {
+                uint32_t q[16];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const uint4 v = live ? __ldg(src + c4 * 4 + i) : make_uint4(0, 0, 0, 0);
-                    r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+                    q[4 * i] = v.x; q[4 * i + 1] = v.y; q[4 * i + 2] = v.z; q[4 * i + 3] = v.w;
                 }
-                tmem_st16(lane_base + TQ + c4 * 16, r);
+                tmem_st16(lane_base + TQ + grp * 32 + c4 * 16, q);
             }
             tmem_wait_st();
             fence_before();
-            mbar_arrive(bar(B_QFULL));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_QFULL));
         }
+        // First tile in which this row may see a key (lists only, so uniform over the query
+        // block): the group that owns that tile fixes the row's softmax reference there and
+        // publishes it; the other group picks it up before its first later tile.
+        int tref = T;
+        for (int sl = 0; sl < nU; ++sl)
+            if ((s_list[sl] >> side) & 1) { tref = sl >> 1; break; }
         float nref = 0.f;         // minus the softmax reference (base-2, scaled)
         bool have_ref = false;
-        float lr = 0.f;           // sum of the rounded weights of this row
+        float lr = 0.f;           // sum of the rounded weights this thread produced for its row
         bool ok = true;
-        for (int t = 0; t < T; ++t) {
-            const int sb = t & 1;
-            if (!mbar_wait(bar(B_SFULL + sb), (t >> 1) & 1, s_abort, a.status, 0x80)) { ok = false; break; }
+        const uint32_t sbase = lane_base + TS + grp * 128;   // group g owns S/P buffer g
+        for (int t = grp; t < T; t += 2) {
+            const int e0 = s_list[2 * t];
+            const int e1 = (2 * t + 1 < nU) ? s_list[2 * t + 1] : 0;
+            const bool mine0 = (e0 >> side) & 1, mine1 = (e1 >> side) & 1;
+            const int nv0 = N - (e0 >> 2) * USV_BLOCK;   // keys of the block with index < N
+            const int nv1 = N - (e1 >> 2) * USV_BLOCK;
+            if (!mbar_wait(bar(B_SFULL + grp), (t >> 1) & 1, s_abort, a.status, 0x80)) { ok = false; break; }
             fence_after();
-            const uint32_t sbase = lane_base + TS + sb * 128;
-#pragma unroll
-            for (int hb = 0; hb < 2; ++hb) {
-                const int slot = 2 * t + hb;
-                const int e = slot < nU ? s_list[slot] : 0;
-                const bool mine = (e >> side) & 1;
-                if (mine) {
-                    const int nvalid = N - (e >> 2) * USV_BLOCK;   // keys of this block with index < N
-                    uint32_t s0[32], s1[32];
-                    tmem_ld32(sbase + hb * 64, s0);
-                    tmem_ld32(sbase + hb * 64 + 32, s1);
+            uint32_t s0[32], s1[32], s2[32], s3[32];
+            if (mine0) {
+                tmem_ld32(sbase, s0);
+                tmem_ld32(sbase + 32, s1);
+            }
+            if (mine1) {
+                tmem_ld32(sbase + 64, s2);
+                tmem_ld32(sbase + 96, s3);
+            }
+            if (!have_ref && t >= tref) {
+                if (t == tref) {
                     tmem_wait_ld();
-                    if (!have_ref) {
-                        float mx = -INFINITY;
+                    float mx = -INFINITY;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (j < nvalid) mx = fmaxf(mx, __uint_as_float(s0[j]));
-                            if (j + 32 < nvalid) mx = fmaxf(mx, __uint_as_float(s1[j]));
-                        }
-                        nref = -mx * c;
-                        have_ref = true;
+                    for (int j = 0; j < 32; ++j) {
+                        if (mine0 && j < nv0) mx = fmaxf(mx, __uint_as_float(s0[j]));
+                        if (mine0 && j + 32 < nv0) mx = fmaxf(mx, __uint_as_float(s1[j]));
+                        if (mine1 && j < nv1) mx = fmaxf(mx, __uint_as_float(s2[j]));
+                        if (mine1 && j + 32 < nv1) mx = fmaxf(mx, __uint_as_float(s3[j]));
                     }
-                    uint32_t pk[16];
-                    if (nvalid >= USV_BLOCK) {
-                        lr += weights32<false>(s0, pk, c, nref, 0, nvalid);
-                        tmem_st16(sbase + hb * 32, pk);
-                        lr += weights32<false>(s1, pk, c, nref, 32, nvalid);
-                        tmem_st16(sbase + hb * 32 + 16, pk);
-                    } else {
-                        lr += weights32<true>(s0, pk, c, nref, 0, nvalid);
-                        tmem_st16(sbase + hb * 32, pk);
-                        lr += weights32<true>(s1, pk, c, nref, 32, nvalid);
-                        tmem_st16(sbase + hb * 32 + 16, pk);
-                    }
+                    nref = mx == -INFINITY ? 0.f : -mx * c;
+                    s_max[r] = nref;
+                    mbar_arrive(bar(B_REF + side));
                 } else {
-                    uint32_t z[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) z[j] = 0u;
-                    tmem_st16(sbase + hb * 32, z);
-                    tmem_st16(sbase + hb * 32 + 16, z);
+                    if (!mbar_wait(bar(B_REF + side), 0, s_abort, a.status, 0x400)) { ok = false; break; }
+                    nref = s_max[r];
                 }
+                have_ref = true;
+            }
+            // P of a key block overwrites the first 32 of the 64 logit columns just read
+            uint32_t pk[16];
+            tmem_wait_ld();
+            if (mine0) {
+                if (nv0 >= USV_BLOCK) {
+                    lr += weights32<false>(s0, pk, c, nref, 0, nv0);
+                    tmem_st16(sbase, pk);
+                    lr += weights32<false>(s1, pk, c, nref, 32, nv0);
+                    tmem_st16(sbase + 16, pk);
+                } else {
+                    lr += weights32<true>(s0, pk, c, nref, 0, nv0);
+                    tmem_st16(sbase, pk);
+                    lr += weights32<true>(s1, pk, c, nref, 32, nv0);
+                    tmem_st16(sbase + 16, pk);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[j] = 0u;
+                tmem_st16(sbase, pk);
+                tmem_st16(sbase + 16, pk);
+            }
+            if (mine1) {
+                if (nv1 >= USV_BLOCK) {
+                    lr += weights32<false>(s2, pk, c, nref, 0, nv1);
+                    tmem_st16(sbase + 64, pk);
+                    lr += weights32<false>(s3, pk, c, nref, 32, nv1);
+                    tmem_st16(sbase + 80, pk);
+                } else {
+                    lr += weights32<true>(s2, pk, c, nref, 0, nv1);
+                    tmem_st16(sbase + 64, pk);
+                    lr += weights32<true>(s3, pk, c, nref, 32, nv1);
+                    tmem_st16(sbase + 80, pk);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[j] = 0u;
+                tmem_st16(sbase + 64, pk);
+                tmem_st16(sbase + 80, pk);
             }
             tmem_wait_st();
             fence_before();
-            mbar_arrive(bar(B_PFULL + sb));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_PFULL + grp));
         }
         // ---- epilogue
         if (ok) ok = mbar_wait(bar(B_OFULL), 0, s_abort, a.status, 0x200);
         if (ok) {
             fence_after();
-            const bool in_range = lr > 7.9e-31f && lr < 1.2e30f;   // ~[2^-100, 2^100]
+            s_sum[grp * 128 + r] = lr;
+            mbar_arrive(bar(B_EPI));
+            ok = mbar_wait(bar(B_EPI), 0, s_abort, a.status, 0x800);
+        }
+        if (ok) {
+            const float l = s_sum[r] + s_sum[128 + r];
+            const bool in_range = l > 7.9e-31f && l < 1.2e30f;   // ~[2^-100, 2^100]
             if (live && !in_range) s_flag[side] = 1;
-            const float inv = lr > 0.f ? 1.0f / lr : 0.f;
-            if (a.lse != nullptr && live)
-                a.lse[((int64_t)b * a.H + h) * N + row] = (log2f(lr) - nref) * 0.69314718055994531f;
-            float* o32 = (a.o_f32 != nullptr && live) ? a.o_f32 + (((int64_t)b * a.H + h) * N + row) * D : nullptr;
+            const float inv = l > 0.f ? 1.0f / l : 0.f;
+            if (a.lse != nullptr && live && grp == 0)
+                a.lse[((int64_t)b * a.H + h) * N + row] =
+                    (log2f(l) - (tref < T ? s_max[r] : 0.f)) * 0.69314718055994531f;
+            float* o32 = (a.o_f32 != nullptr && live)
+                             ? a.o_f32 + (((int64_t)b * a.H + h) * N + row) * D + grp * 64 : nullptr;
             unsigned char* stage = sm + SM_K;   // [128 rows][256 B], 16-byte chunks XOR-swizzled by row
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
+            for (int ch = 0; ch < 2; ++ch) {
                 uint32_t orr[32];
-                tmem_ld32(lane_base + TO + ch * 32, orr);
+                tmem_ld32(lane_base + TO + grp * 64 + ch * 32, orr);
                 tmem_wait_ld();
                 float f[32];
 #pragma unroll
@@ -358,20 +433,24 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int cc = ch * 4 + i;
-                    *reinterpret_cast<uint4*>(stage + tid * 256 + ((cc ^ (tid & 15)) << 4)) = float8_to_bf16x8(f + 8 * i);
+                    const int cc = grp * 8 + ch * 4 + i;
+                    *reinterpret_cast<uint4*>(stage + r * 256 + ((cc ^ (r & 15)) << 4)) = float8_to_bf16x8(f + 8 * i);
                 }
             }
-            softmax_bar();
+            mbar_arrive(bar(B_EPI + 1));
+            ok = mbar_wait(bar(B_EPI + 1), 0, s_abort, a.status, 0x1000);
+        }
+        if (ok) {
+            unsigned char* stage = sm + SM_K;
             __nv_bfloat16* O = a.o + b * a.so.sb + h * a.so.sh;
 #pragma unroll 4
-            for (int idx = tid; idx < 128 * 16; idx += 128) {
-                const int r = idx >> 4, cc = idx & 15;
-                const int Ir = r < 64 ? IA : IB;
-                const int grow = Ir * USV_BLOCK + (r & 63);
+            for (int idx = threadIdx.x; idx < 128 * 16; idx += NSOFT) {
+                const int rr = idx >> 4, cc = idx & 15;
+                const int Ir = rr < 64 ? IA : IB;
+                const int grow = Ir * USV_BLOCK + (rr & 63);
                 if (Ir >= 0 && grow < N)
                     *reinterpret_cast<uint4*>(O + (int64_t)grow * a.so.sn + cc * 8) =
-                        *reinterpret_cast<const uint4*>(stage + r * 256 + ((cc ^ (r & 15)) << 4));
+                        *reinterpret_cast<const uint4*>(stage + rr * 256 + ((cc ^ (rr & 15)) << 4));
             }
         }
     }
@@ -394,14 +473,14 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
         // no valid key block at all: defined output (zeros), as the exact kernel does
         __nv_bfloat16* O = a.o + b * a.so.sb + h * a.so.sh;
         for (int idx = threadIdx.x; idx < 128 * (D / 8); idx += blockDim.x) {
-            const int r = idx / (D / 8);
-            const int Ir = r < 64 ? IA : IB;
-            const int grow = Ir * USV_BLOCK + (r & 63);
+            const int rr = idx / (D / 8);
+            const int Ir = rr < 64 ? IA : IB;
+            const int grow = Ir * USV_BLOCK + (rr & 63);
             if (Ir >= 0 && grow < N)
                 *reinterpret_cast<uint4*>(O + (int64_t)grow * a.so.sn + (idx % (D / 8)) * 8) = make_uint4(0, 0, 0, 0);
         }
     }
-    if (warp == 5) {
+    if (warp == W_MMA) {
         fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
     }
@@ -423,7 +502,7 @@ int launch_attn_pair(const AttnArgs& a, int d, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(pr::attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)pr::SMEM_BYTES);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: smem attribute: %s", cudaGetErrorString(e));
-    pr::attn_pair_kernel<<<(unsigned)grid, 192, pr::SMEM_BYTES, st>>>(a, maps);
+    pr::attn_pair_kernel<<<(unsigned)grid, pr::NTHREADS, pr::SMEM_BYTES, st>>>(a, maps);
     USV_CHECK_LAUNCH("attn_pair_kernel");
     return USV_OK;
 }

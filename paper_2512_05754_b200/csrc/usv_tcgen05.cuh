@@ -41,11 +41,15 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
 // device status word.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           unsigned int* status, unsigned int code) {
-    if (mbar_try(bar, parity)) return true;
+    // fast path: plain polling (each try may itself block for a short, hardware-defined time)
+#pragma unroll 1
+    for (int i = 0; i < 2048; ++i)
+        if (mbar_try(bar, parity)) return true;
+    // slow path: keep polling against a wall-clock limit
     const unsigned long long t0 = gtime();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 64; ++i)
+        for (int i = 0; i < 256; ++i)
             if (mbar_try(bar, parity)) return true;
         if (*abort_flag) return false;
         if (gtime() - t0 > WAIT_LIMIT_NS) {
@@ -54,6 +58,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             return false;
         }
     }
+}
+
+// True in exactly one lane of a converged warp.  Single-thread instructions (TMA, MMA, commit)
+// are issued under it from warp-uniform code, so that their operands stay in uniform registers.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred = 0;
+    asm volatile(
+        "{\n\t.reg .b32 rx;\n\t.reg .pred px;\n\t"
+        "elect.sync rx|px, %1;\n\t"
+        "@px mov.s32 %0, 1;\n\t}"
+        : "+r"(pred) : "r"(0xffffffffu));
+    return pred != 0;
 }
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
