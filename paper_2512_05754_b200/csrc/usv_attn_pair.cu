@@ -20,12 +20,18 @@
 // logits.  Rows whose sum leaves [2^-100, 2^100] are reported in a list and recomputed by the
 // exact online-softmax kernel, so the result never depends on that assumption.
 //
-// CTA = 10 warps: warps 0-7 softmax/epilogue as two warpgroups that share the rows (thread i of
-// either group <-> TMEM lane i) and alternate tiles (group g: tiles t = g mod 2, S/P buffer g),
-// so that the load-exponentiate-store chains of two tiles overlap; warp 8 TMA producer, warp 9
-// MMA issuer and TMEM owner.  P overwrites part of the S buffer it came from.
-// All waits are bounded; a wait that gives up sets the device status word and every role leaves
-// its loop.
+// CTA = 18 warps.  Warps 0-15 are four softmax/epilogue warpgroups that share the 128 rows
+// (thread r of every group <-> TMEM lane r <-> query row r).  Group g works on the tiles of
+// parity g >> 1 (S/P buffer g >> 1) and there on key block g & 1 of the tile (64 logit columns),
+// so two tiles are in the softmax stage at a time, each spread over 256 threads.  Warp 16 is the
+// TMA producer, warp 17 the MMA issuer and TMEM owner.  P overwrites the first half of the 64
+// logit columns it came from.
+//
+// The MMA issuer commits once per tile, on the barrier that publishes S(t).  MMAs execute in
+// issue order, so that arrival also says that every MMA issued before S(t) is complete; the
+// softmax threads that see it hand the K stage of tile t and the V stage of tile t - 2 back to
+// the producer.  All waits are bounded; a wait that gives up sets the device status word and
+// every role leaves its loop.
 #include "usv_attn.cuh"
 #include "usv_tcgen05.cuh"
 
@@ -36,56 +42,60 @@ namespace pr {
 using namespace t5;
 
 constexpr int D = 128;
-constexpr int STAGES = 3;                       // K and V tile stages
+constexpr int KT = 2 * USV_BLOCK;               // keys per tile = two key blocks
+constexpr int NWG = 4;                          // softmax warpgroups
+constexpr int KSTAGES = 2;                      // K tile stages (freed as soon as S is computed)
+constexpr int VSTAGES = 4;                      // V tile stages (freed one tile after P.V is issued)
 constexpr int MAX_NB = 4096;                    // key blocks per sequence this kernel covers
-constexpr uint32_t TILE_BYTES = 128 * D * 2;    // 32 KB: two 64-key blocks, [d-half][128 keys][128 B]
+constexpr uint32_t TILE_BYTES = KT * D * 2;     // 32 KB: [d-half][128 keys][128 B]
 constexpr uint32_t SM_K = 0;
-constexpr uint32_t SM_V = SM_K + STAGES * TILE_BYTES;
-constexpr uint32_t SM_BAR = SM_V + STAGES * TILE_BYTES;
+constexpr uint32_t SM_V = SM_K + KSTAGES * TILE_BYTES;
+constexpr uint32_t SM_BAR = SM_V + VSTAGES * TILE_BYTES;
 // barrier slots (8 bytes each)
-enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = B_KFULL + STAGES, B_VFULL = B_KEMPTY + STAGES,
-       B_VEMPTY = B_VFULL + STAGES, B_SFULL = B_VEMPTY + STAGES, B_PFULL = B_SFULL + 2,
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = B_KFULL + KSTAGES, B_VFULL = B_KEMPTY + KSTAGES,
+       B_VEMPTY = B_VFULL + VSTAGES, B_SFULL = B_VEMPTY + VSTAGES, B_PFULL = B_SFULL + 2,
        B_OFULL = B_PFULL + 2, B_REF, B_EPI = B_REF + 2, B_COUNT = B_EPI + 2 };
 static_assert(B_COUNT <= 32, "barrier area");
 constexpr uint32_t SM_MISC = SM_BAR + 8 * 32;            // tmem base, abort flag, flags, union size
 constexpr uint32_t SM_BITS = SM_MISC + 64;               // two bitmaps of MAX_NB bits
 constexpr uint32_t SM_LIST = SM_BITS + 2 * (MAX_NB / 8); // int[MAX_NB]: (key block << 2) | in-A | in-B << 1
-constexpr uint32_t SM_MAX = SM_LIST + MAX_NB * 4;        // float[128 rows] minus the softmax reference (+ spare)
-constexpr uint32_t SM_SUM = SM_MAX + 2 * 128 * 4;        // float[2 groups][128 rows] row sums
-constexpr uint32_t SM_TOTAL = SM_SUM + 2 * 128 * 4;
+constexpr uint32_t SM_REFV = SM_LIST + MAX_NB * 4;       // float[128]: minus the softmax reference per row
+constexpr uint32_t SM_SUM = SM_REFV + 128 * 4;           // float[NWG][128]: partial row sums
+constexpr uint32_t SM_TOTAL = SM_SUM + NWG * 128 * 4;
 constexpr size_t SMEM_BYTES = SM_TOTAL + 1024;           // + slack for 1024-byte alignment
 
 // TMEM columns: Q (bf16 pairs) | S/P buffer 0 | S/P buffer 1 | O
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t TQ = 0, TS = 64, TO = 320;
+constexpr uint32_t TQ = 0, TS = 64, TO = TS + 2 * 128;
+static_assert(TO + 128 <= TMEM_COLS, "TMEM budget");
 
-constexpr int NSOFT = 256;   // softmax threads
+constexpr int NSOFT = NWG * 128;   // softmax threads
 constexpr int NTHREADS = NSOFT + 64;
-__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+constexpr int W_TMA = NSOFT / 32, W_MMA = NSOFT / 32 + 1;
+__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory"); }
 
 struct Maps {
     CUtensorMap k, v;
 };
 
-// exp2 of 32 scaled logits -> 16 packed bf16 pairs; returns the sum of the ROUNDED weights
+// exp2 of 32 scaled logits -> 16 packed bf16 pairs; adds the (unrounded) weights to the two
+// lanes of `acc`.  Two logits at a time on the packed-fp32 pipe.
 template <bool MASKED>
-__device__ __forceinline__ float weights32(const uint32_t* sr, uint32_t* pk, float c, float nref, int col0,
-                                           int nvalid) {
-    float acc0 = 0.f, acc1 = 0.f;
+__device__ __forceinline__ void weights32(const uint32_t* sr, uint32_t* pk, uint64_t c2, uint64_t nref2, int col0,
+                                          int nvalid, uint64_t& acc) {
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        float p0 = ex2(fmaf(__uint_as_float(sr[2 * j]), c, nref));
-        float p1 = ex2(fmaf(__uint_as_float(sr[2 * j + 1]), c, nref));
+        const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(sr[2 * j]), __uint_as_float(sr[2 * j + 1])), c2, nref2);
+        float x0, x1;
+        unpack_f32x2(x2, x0, x1);
+        float p0 = ex2(x0), p1 = ex2(x1);
         if (MASKED) {
             if (col0 + 2 * j >= nvalid) p0 = 0.f;
             if (col0 + 2 * j + 1 >= nvalid) p1 = 0.f;
         }
-        const uint32_t w = pack_bf16x2(p0, p1);
-        acc0 += __uint_as_float(w << 16);
-        acc1 += __uint_as_float(w & 0xffff0000u);
-        pk[j] = w;
+        acc = add_f32x2(acc, pack_f32x2(p0, p1));
+        pk[j] = pack_bf16x2(p0, p1);
     }
-    return acc0 + acc1;
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -101,7 +111,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     volatile int* s_nu = reinterpret_cast<volatile int*>(sm + SM_MISC + 16);
     uint32_t* s_bits = reinterpret_cast<uint32_t*>(sm + SM_BITS);
     int* s_list = reinterpret_cast<int*>(sm + SM_LIST);
-    float* s_max = reinterpret_cast<float*>(sm + SM_MAX);
+    float* s_refv = reinterpret_cast<float*>(sm + SM_REFV);
     float* s_sum = reinterpret_cast<float*>(sm + SM_SUM);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -115,28 +125,37 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const int IA = 2 * pair;
     const int IB = (2 * pair + 1 < NB) ? 2 * pair + 1 : -1;
     const int nwords = (NB + 31) >> 5;
-    constexpr int W_TMA = NSOFT / 32, W_MMA = NSOFT / 32 + 1;
 
-    // ---- set-up: barriers, TMEM, ascending union of the two selection rows
+    // softmax-thread geometry (meaningful for warps < W_TMA)
+    const int grp = warp >> 2;                       // tiles of parity grp >> 1, key block grp & 1
+    const int r = threadIdx.x & 127;                 // query row within the pair, = TMEM lane
+    const int side = r >> 6;                         // 0: block A, 1: block B (uniform per warp)
+    const int Iq = side ? IB : IA;
+    const int row = Iq * USV_BLOCK + (r & 63);
+    const bool live = Iq >= 0 && row < N;
+
+    // ---- set-up: barriers, TMEM, ascending union of the two selection rows, Q -> TMEM
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), NSOFT / 32);       // one arrival per softmax warp
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < KSTAGES; ++s) {
             mbar_init(bar(B_KFULL + s), 1);
             mbar_init(bar(B_KEMPTY + s), 1);
+        }
+        for (int s = 0; s < VSTAGES; ++s) {
             mbar_init(bar(B_VFULL + s), 1);
             mbar_init(bar(B_VEMPTY + s), 1);
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(B_SFULL + s), 1);
-            mbar_init(bar(B_PFULL + s), 4);         // one arrival per warp of the group
+            mbar_init(bar(B_PFULL + s), 8);         // one arrival per warp of the two groups
         }
         mbar_init(bar(B_OFULL), 1);
         // rendezvous of the softmax threads after the first bounded wait: mbarriers, so that they
         // too can give up (a bar.sync would hang if one thread had left its loop)
-        mbar_init(bar(B_REF), 64);
-        mbar_init(bar(B_REF + 1), 64);
-        mbar_init(bar(B_EPI), NSOFT);
-        mbar_init(bar(B_EPI + 1), NSOFT);
+        mbar_init(bar(B_REF), 2);                   // the two warps of the owning group on a side
+        mbar_init(bar(B_REF + 1), 2);
+        mbar_init(bar(B_EPI), NSOFT / 32);
+        mbar_init(bar(B_EPI + 1), NSOFT / 32);
         *s_abort = 0;
         s_flag[0] = 0;
         s_flag[1] = 0;
@@ -147,15 +166,26 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                      ::"r"(base + SM_MISC), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    uint32_t* bitsA = s_bits;
+    uint32_t* bitsB = s_bits + MAX_NB / 32;
+    uint4 qv[4];   // this thread's quarter of its query row (32 of the 128 bf16)
     if (warp < W_TMA) {
-        const int tid = threadIdx.x;
-        uint32_t* bitsA = s_bits;
-        uint32_t* bitsB = s_bits + MAX_NB / 32;
-        for (int w = tid; w < nwords; w += NSOFT) {
+        const uint4* src = reinterpret_cast<const uint4*>(a.q + b * a.sq.sb + h * a.sq.sh +
+                                                          (int64_t)row * a.sq.sn + grp * 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) qv[i] = live ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
+        for (int w = threadIdx.x; w < nwords; w += NSOFT) {
             bitsA[w] = 0;
             bitsB[w] = 0;
         }
-        softmax_bar();
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = *s_tmem;
+    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    if (warp < W_TMA) {
+        const int tid = threadIdx.x;
         const int32_t* selA = a.sel + (((int64_t)b * a.H + h) * NB + IA) * a.kmax;
         for (int t = tid; t < kh; t += NSOFT) {
             const int J = selA[t];
@@ -168,6 +198,17 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 if (J >= 0 && J < NB) atomicOr(&bitsB[J >> 5], 1u << (J & 31));
             }
         }
+        // this thread's part of its query row -> TMEM (two bf16 of consecutive d per column)
+        uint32_t q[16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            q[4 * i] = qv[i].x; q[4 * i + 1] = qv[i].y; q[4 * i + 2] = qv[i].z; q[4 * i + 3] = qv[i].w;
+        }
+        tmem_st16(lane_base + TQ + grp * 16, q);
+        tmem_wait_st();
+        fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(B_QFULL));
         softmax_bar();
         if (warp == 0) {
             int running = 0;
@@ -188,18 +229,15 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
             if (lane == 0) *s_nu = running;
         }
     }
-    fence_before();
     __syncthreads();
-    fence_after();
-    const uint32_t tmem = *s_tmem;
     const int nU = *s_nu;
     const int T = (nU + 1) >> 1;   // 128-key tiles
 
     if (warp == W_TMA) {
         // ================= TMA producer (whole warp in the loop, one elected lane issues) ======
         for (int t = 0; t < T; ++t) {
-            const int s = t % STAGES;
-            const uint32_t ph = (t / STAGES) & 1;
+            const int s = t % KSTAGES, sv = t % VSTAGES;
+            const uint32_t ph = (t / KSTAGES) & 1, phv = (t / VSTAGES) & 1;
             const int J0 = s_list[2 * t] >> 2;
             const int J1 = (2 * t + 1 < nU) ? (s_list[2 * t + 1] >> 2) : J0;  // odd tail: finite filler, masked
             if (!mbar_wait(bar(B_KEMPTY + s), ph ^ 1, s_abort, a.status, 0x1)) break;
@@ -212,31 +250,33 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 tma_load_4d(kd + 24576, &maps.k, bar(B_KFULL + s), 64, J1 * USV_BLOCK, h, b);
             }
             __syncwarp();
-            if (!mbar_wait(bar(B_VEMPTY + s), ph ^ 1, s_abort, a.status, 0x2)) break;
-            const uint32_t vd = base + SM_V + s * TILE_BYTES;
+            if (!mbar_wait(bar(B_VEMPTY + sv), phv ^ 1, s_abort, a.status, 0x2)) break;
+            const uint32_t vd = base + SM_V + sv * TILE_BYTES;
             if (elect_one()) {
-                mbar_expect_tx(bar(B_VFULL + s), TILE_BYTES);
-                tma_load_4d(vd, &maps.v, bar(B_VFULL + s), 0, J0 * USV_BLOCK, h, b);
-                tma_load_4d(vd + 8192, &maps.v, bar(B_VFULL + s), 0, J1 * USV_BLOCK, h, b);
-                tma_load_4d(vd + 16384, &maps.v, bar(B_VFULL + s), 64, J0 * USV_BLOCK, h, b);
-                tma_load_4d(vd + 24576, &maps.v, bar(B_VFULL + s), 64, J1 * USV_BLOCK, h, b);
+                mbar_expect_tx(bar(B_VFULL + sv), TILE_BYTES);
+                tma_load_4d(vd, &maps.v, bar(B_VFULL + sv), 0, J0 * USV_BLOCK, h, b);
+                tma_load_4d(vd + 8192, &maps.v, bar(B_VFULL + sv), 0, J1 * USV_BLOCK, h, b);
+                tma_load_4d(vd + 16384, &maps.v, bar(B_VFULL + sv), 64, J0 * USV_BLOCK, h, b);
+                tma_load_4d(vd + 24576, &maps.v, bar(B_VFULL + sv), 64, J1 * USV_BLOCK, h, b);
             }
             __syncwarp();
         }
     } else if (warp == W_MMA) {
         // ================= MMA issuer (whole warp in the loop, one elected lane issues) ========
         if (T > 0) {
-            constexpr uint32_t IDESC_S = instr_desc(128, 128, 0, 0);   // Q (TMEM) x K (K-major)
-            constexpr uint32_t IDESC_O = instr_desc(128, 128, 0, 1);   // P (TMEM) x V (MN-major)
+            constexpr uint32_t IDESC_S = instr_desc(128, KT, 0, 0);    // Q (TMEM) x K (K-major)
+            constexpr uint32_t IDESC_O = instr_desc(128, D, 0, 1);     // P (TMEM) x V (MN-major)
             const uint64_t kdesc0 = smem_desc(base + SM_K, 16, 1024);       // + byte offset >> 4
             const uint64_t vdesc0 = smem_desc(base + SM_V, 16384, 1024);
             bool ok = mbar_wait(bar(B_QFULL), 0, s_abort, a.status, 0x4);
-            auto issue_s = [&](int t) -> bool {
-                const int s = t % STAGES;
-                const uint32_t ph = (t / STAGES) & 1;
+            fence_after();
+            // S(t) -> buffer t & 1.  The MMA that last read P from that buffer, PV(t - 2), has been
+            // issued by the time S(t) is (see the loop), and MMAs execute in issue order.
+            auto issue_s = [&](int t, bool k_ready) -> bool {
+                const int s = t % KSTAGES;
+                const uint32_t ph = (t / KSTAGES) & 1;
                 const int sb = t & 1;
-                if (!mbar_wait(bar(B_KFULL + s), ph, s_abort, a.status, 0x8)) return false;
-                fence_after();
+                if (!k_ready && !mbar_wait(bar(B_KFULL + s), ph, s_abort, a.status, 0x8)) return false;
                 const uint64_t kdesc = kdesc0 + ((s * TILE_BYTES) >> 4);
                 const uint32_t d_s = tmem + TS + sb * 128;
                 if (elect_one()) {
@@ -244,129 +284,105 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                     for (int ks = 0; ks < D / 16; ++ks)
                         umma_ts(d_s, tmem + TQ + ks * 8, kdesc + (((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
                                 IDESC_S, ks > 0);
-                    umma_commit(bar(B_KEMPTY + s));
                     umma_commit(bar(B_SFULL + sb));
                 }
-                __syncwarp();
                 return true;
             };
-            if (ok) ok = issue_s(0);
+            if (ok) ok = issue_s(0, false);
             for (int t = 0; ok && t < T; ++t) {
-                // S of the next tile goes to the other buffer; the MMA before it that read P from
-                // there (tile t-1) was issued earlier by the same lane, and MMAs execute in order.
-                if (t + 1 < T) {
-                    ok = issue_s(t + 1);
+                const int sv = t % VSTAGES;
+                const uint32_t phv = (t / VSTAGES) & 1;
+                const int sb = t & 1;
+                // poll the three barriers of this step together: their latencies overlap
+                const int t1 = t + 1;
+                const bool k_rdy = t1 < T && mbar_try(bar(B_KFULL + t1 % KSTAGES), (t1 / KSTAGES) & 1);
+                const bool v_rdy = mbar_try(bar(B_VFULL + sv), phv);
+                const bool p_rdy = mbar_try(bar(B_PFULL + sb), (t >> 1) & 1);
+                if (t1 < T) {
+                    ok = issue_s(t1, k_rdy);   // early: the softmax of tile t + 1 overlaps PV(t)
                     if (!ok) break;
                 }
-                const int s = t % STAGES;
-                const uint32_t ph = (t / STAGES) & 1;
-                const int sb = t & 1;
-                if (!mbar_wait(bar(B_VFULL + s), ph, s_abort, a.status, 0x20)) break;
-                if (!mbar_wait(bar(B_PFULL + sb), (t >> 1) & 1, s_abort, a.status, 0x40)) break;
+                if (!v_rdy && !mbar_wait(bar(B_VFULL + sv), phv, s_abort, a.status, 0x20)) break;
+                if (!p_rdy && !mbar_wait(bar(B_PFULL + sb), (t >> 1) & 1, s_abort, a.status, 0x40)) break;
                 fence_after();
-                const uint64_t vdesc = vdesc0 + ((s * TILE_BYTES) >> 4);
+                const uint64_t vdesc = vdesc0 + ((sv * TILE_BYTES) >> 4);
                 const uint32_t a_p = tmem + TS + sb * 128;
                 if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        umma_ts(tmem + TO, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vdesc + ((ks * 2048) >> 4),
-                                IDESC_O, (t > 0 || ks > 0));
-                    umma_commit(bar(B_VEMPTY + s));
+                    for (int ks = 0; ks < KT / 16; ++ks)
+                        umma_ts(tmem + TO, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vdesc + ((ks * 2048) >> 4), IDESC_O,
+                                (t > 0 || ks > 0));
                     if (t == T - 1) umma_commit(bar(B_OFULL));
                 }
-                __syncwarp();
             }
         }
     } else if (T > 0) {
-        // ===== softmax + epilogue: thread r of either group <-> TMEM lane r <-> query row r =====
-        const int grp = warp >> 2;                       // key block of each tile this group handles
-        const int r = threadIdx.x & 127;
-        const int side = r >> 6;                         // 0: block A, 1: block B (uniform per warp)
-        const int Iq = side ? IB : IA;
-        const int row = Iq * USV_BLOCK + (r & 63);
-        const bool live = Iq >= 0 && row < N;
-        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        // ===== softmax + epilogue =====
         const float c = a.scale_log2;
-        {
-            // this thread's half of its query row -> TMEM (two bf16 of consecutive d per column)
-            const uint4* src = reinterpret_cast<const uint4*>(a.q + b * a.sq.sb + h * a.sq.sh +
-                                                              (int64_t)row * a.sq.sn + grp * 64);
-#pragma unroll
-            for (int c4 = 0; c4 < 2; ++c4) {
-                uint32_t q[16];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint4 v = live ? __ldg(src + c4 * 4 + i) : make_uint4(0, 0, 0, 0);
-                    q[4 * i] = v.x; q[4 * i + 1] = v.y; q[4 * i + 2] = v.z; q[4 * i + 3] = v.w;
-                }
-                tmem_st16(lane_base + TQ + grp * 32 + c4 * 16, q);
-            }
-            tmem_wait_st();
-            fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B_QFULL));
-        }
-        // First tile in which this row may see a key (lists only, so uniform over the query
-        // block): the group that owns that tile fixes the row's softmax reference there and
-        // publishes it; the other group picks it up before its first later tile.
-        int tref = T;
+        // First union slot whose key block this row may see (lists only, so uniform over the
+        // query block): the group that owns that slot fixes the row's softmax reference there
+        // and publishes it; the other groups pick it up before their first later slot.
+        int sref = nU;
         for (int sl = 0; sl < nU; ++sl)
-            if ((s_list[sl] >> side) & 1) { tref = sl >> 1; break; }
+            if ((s_list[sl] >> side) & 1) { sref = sl; break; }
+        const int tp = grp >> 1, hb = grp & 1;
         float nref = 0.f;         // minus the softmax reference (base-2, scaled)
         bool have_ref = false;
-        float lr = 0.f;           // sum of the rounded weights this thread produced for its row
+        uint64_t lr2 = 0;         // two partial sums of the weights this thread produced for its row
+        uint64_t nref2 = 0;
+        const uint64_t c2 = pack_f32x2(c, c);
         bool ok = true;
-        const uint32_t sbase = lane_base + TS + grp * 128;   // group g owns S/P buffer g
-        for (int t = grp; t < T; t += 2) {
-            const int e0 = s_list[2 * t];
-            const int e1 = (2 * t + 1 < nU) ? s_list[2 * t + 1] : 0;
-            const bool mine0 = (e0 >> side) & 1, mine1 = (e1 >> side) & 1;
-            const int nv0 = N - (e0 >> 2) * USV_BLOCK;   // keys of the block with index < N
-            const int nv1 = N - (e1 >> 2) * USV_BLOCK;
-            if (!mbar_wait(bar(B_SFULL + grp), (t >> 1) & 1, s_abort, a.status, 0x80)) { ok = false; break; }
+        const uint32_t sbase = lane_base + TS + tp * 128 + hb * 64;
+        for (int t = tp; t < T; t += 2) {
+            const int slot = 2 * t + hb;
+            const int e = slot < nU ? s_list[slot] : 0;
+            const bool mine = (e >> side) & 1;
+            const int nv = N - (e >> 2) * USV_BLOCK;   // keys of the block with index < N
+            if (!mbar_wait(bar(B_SFULL + tp), (t >> 1) & 1, s_abort, a.status, 0x80)) { ok = false; break; }
             fence_after();
-            uint32_t s0[32], s1[32], s2[32], s3[32];
-            if (mine0) {
+            if (hb == 0 && (warp & 3) == 0 && lane == 0) {
+                // S(t) is complete, and so is every MMA issued before it: PV(t - 2) and older
+                mbar_arrive(bar(B_KEMPTY + t % KSTAGES));
+                if (t >= 2) mbar_arrive(bar(B_VEMPTY + (t - 2) % VSTAGES));
+            }
+            uint32_t s0[32], s1[32];
+            if (mine) {
                 tmem_ld32(sbase, s0);
                 tmem_ld32(sbase + 32, s1);
             }
-            if (mine1) {
-                tmem_ld32(sbase + 64, s2);
-                tmem_ld32(sbase + 96, s3);
-            }
-            if (!have_ref && t >= tref) {
-                if (t == tref) {
+            if (!have_ref && slot >= sref) {
+                if (slot == sref) {
                     tmem_wait_ld();
                     float mx = -INFINITY;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        if (mine0 && j < nv0) mx = fmaxf(mx, __uint_as_float(s0[j]));
-                        if (mine0 && j + 32 < nv0) mx = fmaxf(mx, __uint_as_float(s1[j]));
-                        if (mine1 && j < nv1) mx = fmaxf(mx, __uint_as_float(s2[j]));
-                        if (mine1 && j + 32 < nv1) mx = fmaxf(mx, __uint_as_float(s3[j]));
+                        if (j < nv) mx = fmaxf(mx, __uint_as_float(s0[j]));
+                        if (j + 32 < nv) mx = fmaxf(mx, __uint_as_float(s1[j]));
                     }
                     nref = mx == -INFINITY ? 0.f : -mx * c;
-                    s_max[r] = nref;
-                    mbar_arrive(bar(B_REF + side));
+                    s_refv[r] = nref;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(B_REF + side));
                 } else {
                     if (!mbar_wait(bar(B_REF + side), 0, s_abort, a.status, 0x400)) { ok = false; break; }
-                    nref = s_max[r];
+                    nref = s_refv[r];
                 }
+                nref2 = pack_f32x2(nref, nref);
                 have_ref = true;
             }
-            // P of a key block overwrites the first 32 of the 64 logit columns just read
+            // P overwrites the first 32 of the 64 logit columns just read
             uint32_t pk[16];
-            tmem_wait_ld();
-            if (mine0) {
-                if (nv0 >= USV_BLOCK) {
-                    lr += weights32<false>(s0, pk, c, nref, 0, nv0);
+            if (mine) {
+                tmem_wait_ld();
+                if (nv >= USV_BLOCK) {
+                    weights32<false>(s0, pk, c2, nref2, 0, nv, lr2);
                     tmem_st16(sbase, pk);
-                    lr += weights32<false>(s1, pk, c, nref, 32, nv0);
+                    weights32<false>(s1, pk, c2, nref2, 32, nv, lr2);
                     tmem_st16(sbase + 16, pk);
                 } else {
-                    lr += weights32<true>(s0, pk, c, nref, 0, nv0);
+                    weights32<true>(s0, pk, c2, nref2, 0, nv, lr2);
                     tmem_st16(sbase, pk);
-                    lr += weights32<true>(s1, pk, c, nref, 32, nv0);
+                    weights32<true>(s1, pk, c2, nref2, 32, nv, lr2);
                     tmem_st16(sbase + 16, pk);
                 }
             } else {
@@ -375,73 +391,57 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 tmem_st16(sbase, pk);
                 tmem_st16(sbase + 16, pk);
             }
-            if (mine1) {
-                if (nv1 >= USV_BLOCK) {
-                    lr += weights32<false>(s2, pk, c, nref, 0, nv1);
-                    tmem_st16(sbase + 64, pk);
-                    lr += weights32<false>(s3, pk, c, nref, 32, nv1);
-                    tmem_st16(sbase + 80, pk);
-                } else {
-                    lr += weights32<true>(s2, pk, c, nref, 0, nv1);
-                    tmem_st16(sbase + 64, pk);
-                    lr += weights32<true>(s3, pk, c, nref, 32, nv1);
-                    tmem_st16(sbase + 80, pk);
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) pk[j] = 0u;
-                tmem_st16(sbase + 64, pk);
-                tmem_st16(sbase + 80, pk);
-            }
             tmem_wait_st();
             fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B_PFULL + grp));
+            if (lane == 0) mbar_arrive(bar(B_PFULL + tp));
         }
         // ---- epilogue
         if (ok) ok = mbar_wait(bar(B_OFULL), 0, s_abort, a.status, 0x200);
         if (ok) {
             fence_after();
-            s_sum[grp * 128 + r] = lr;
-            mbar_arrive(bar(B_EPI));
+            float lr_lo, lr_hi;
+            unpack_f32x2(lr2, lr_lo, lr_hi);
+            s_sum[grp * 128 + r] = lr_lo + lr_hi;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_EPI));
             ok = mbar_wait(bar(B_EPI), 0, s_abort, a.status, 0x800);
         }
         if (ok) {
-            const float l = s_sum[r] + s_sum[128 + r];
+            float l = 0.f;
+#pragma unroll
+            for (int g = 0; g < NWG; ++g) l += s_sum[g * 128 + r];
             const bool in_range = l > 7.9e-31f && l < 1.2e30f;   // ~[2^-100, 2^100]
             if (live && !in_range) s_flag[side] = 1;
             const float inv = l > 0.f ? 1.0f / l : 0.f;
             if (a.lse != nullptr && live && grp == 0)
                 a.lse[((int64_t)b * a.H + h) * N + row] =
-                    (log2f(l) - (tref < T ? s_max[r] : 0.f)) * 0.69314718055994531f;
+                    (log2f(l) - (sref < nU ? s_refv[r] : 0.f)) * 0.69314718055994531f;
             float* o32 = (a.o_f32 != nullptr && live)
-                             ? a.o_f32 + (((int64_t)b * a.H + h) * N + row) * D + grp * 64 : nullptr;
-            unsigned char* stage = sm + SM_K;   // [128 rows][256 B], 16-byte chunks XOR-swizzled by row
+                             ? a.o_f32 + (((int64_t)b * a.H + h) * N + row) * D + grp * 32 : nullptr;
+            unsigned char* stage = sm + SM_V;   // [128 rows][256 B], 16-byte chunks XOR-swizzled by row
+            uint32_t orr[32];
+            tmem_ld32(lane_base + TO + grp * 32, orr);
+            tmem_wait_ld();
+            float f[32];
 #pragma unroll
-            for (int ch = 0; ch < 2; ++ch) {
-                uint32_t orr[32];
-                tmem_ld32(lane_base + TO + grp * 64 + ch * 32, orr);
-                tmem_wait_ld();
-                float f[32];
+            for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(orr[j]) * inv;
+            if (o32 != nullptr) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(orr[j]) * inv;
-                if (o32 != nullptr) {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        *reinterpret_cast<float4*>(o32 + ch * 32 + j * 4) =
-                            make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int cc = grp * 8 + ch * 4 + i;
-                    *reinterpret_cast<uint4*>(stage + r * 256 + ((cc ^ (r & 15)) << 4)) = float8_to_bf16x8(f + 8 * i);
-                }
+                for (int j = 0; j < 8; ++j)
+                    *reinterpret_cast<float4*>(o32 + j * 4) = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
             }
-            mbar_arrive(bar(B_EPI + 1));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int cc = grp * 4 + i;
+                *reinterpret_cast<uint4*>(stage + r * 256 + ((cc ^ (r & 15)) << 4)) = float8_to_bf16x8(f + 8 * i);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_EPI + 1));
             ok = mbar_wait(bar(B_EPI + 1), 0, s_abort, a.status, 0x1000);
         }
         if (ok) {
-            unsigned char* stage = sm + SM_K;
+            unsigned char* stage = sm + SM_V;
             __nv_bfloat16* O = a.o + b * a.so.sb + h * a.so.sh;
 #pragma unroll 4
             for (int idx = threadIdx.x; idx < 128 * 16; idx += NSOFT) {
