@@ -20,18 +20,18 @@
 // logits.  Rows whose sum leaves [2^-100, 2^100] are reported in a list and recomputed by the
 // exact online-softmax kernel, so the result never depends on that assumption.
 //
-// CTA = 18 warps.  Warps 0-15 are four softmax/epilogue warpgroups that share the 128 rows
+// CTA = 19 warps.  Warps 0-15 are four softmax/epilogue warpgroups that share the 128 rows
 // (thread r of every group <-> TMEM lane r <-> query row r).  Group g works on the tiles of
 // parity g >> 1 (S/P buffer g >> 1) and there on key block g & 1 of the tile (64 logit columns),
 // so two tiles are in the softmax stage at a time, each spread over 256 threads.  Warp 16 is the
-// TMA producer, warp 17 the MMA issuer and TMEM owner.  P overwrites the first half of the 64
-// logit columns it came from.
+// K producer (TMA), warp 17 the MMA issuer and TMEM owner, warp 18 the V producer.
 //
-// The MMA issuer commits once per tile, on the barrier that publishes S(t).  MMAs execute in
-// issue order, so that arrival also says that every MMA issued before S(t) is complete; the
-// softmax threads that see it hand the K stage of tile t and the V stage of tile t - 2 back to
-// the producer.  All waits are bounded; a wait that gives up sets the device status word and
-// every role leaves its loop.
+// TMEM holds Q, two S buffers, O and ONE P buffer.  A softmax thread gives its S buffer back as
+// soon as the logits are in its registers (S of the tile after next is then computed while it
+// exponentiates), and writes P once the P.V product of the tile before has finished reading the
+// P buffer.  There is one commit after S(t) (publishes S, frees the K stage) and one after
+// PV(t) (frees the P buffer and the V stage).  All waits are bounded; a wait that
+// gives up sets the device status word and every role leaves its loop.
 #include "usv_attn.cuh"
 #include "usv_tcgen05.cuh"
 
@@ -44,8 +44,8 @@ using namespace t5;
 constexpr int D = 128;
 constexpr int KT = 2 * USV_BLOCK;               // keys per tile = two key blocks
 constexpr int NWG = 4;                          // softmax warpgroups
-constexpr int KSTAGES = 2;                      // K tile stages (freed as soon as S is computed)
-constexpr int VSTAGES = 4;                      // V tile stages (freed one tile after P.V is issued)
+constexpr int KSTAGES = 3;                      // K tile stages
+constexpr int VSTAGES = 3;                      // V tile stages
 constexpr int MAX_NB = 4096;                    // key blocks per sequence this kernel covers
 constexpr uint32_t TILE_BYTES = KT * D * 2;     // 32 KB: [d-half][128 keys][128 B]
 constexpr uint32_t SM_K = 0;
@@ -53,8 +53,8 @@ constexpr uint32_t SM_V = SM_K + KSTAGES * TILE_BYTES;
 constexpr uint32_t SM_BAR = SM_V + VSTAGES * TILE_BYTES;
 // barrier slots (8 bytes each)
 enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = B_KFULL + KSTAGES, B_VFULL = B_KEMPTY + KSTAGES,
-       B_VEMPTY = B_VFULL + VSTAGES, B_SFULL = B_VEMPTY + VSTAGES, B_PFULL = B_SFULL + 2,
-       B_OFULL = B_PFULL + 2, B_REF, B_EPI = B_REF + 2, B_COUNT = B_EPI + 2 };
+       B_VEMPTY = B_VFULL + VSTAGES, B_SFULL = B_VEMPTY + VSTAGES, B_SFREE = B_SFULL + 2,
+       B_PFULL = B_SFREE + 2, B_PFREE = B_PFULL + 2, B_OFULL = B_PFREE + 2, B_REF, B_EPI = B_REF + 2, B_COUNT = B_EPI + 2 };
 static_assert(B_COUNT <= 32, "barrier area");
 constexpr uint32_t SM_MISC = SM_BAR + 8 * 32;            // tmem base, abort flag, flags, union size
 constexpr uint32_t SM_BITS = SM_MISC + 64;               // two bitmaps of MAX_NB bits
@@ -64,14 +64,14 @@ constexpr uint32_t SM_SUM = SM_REFV + 128 * 4;           // float[NWG][128]: par
 constexpr uint32_t SM_TOTAL = SM_SUM + NWG * 128 * 4;
 constexpr size_t SMEM_BYTES = SM_TOTAL + 1024;           // + slack for 1024-byte alignment
 
-// TMEM columns: Q (bf16 pairs) | S/P buffer 0 | S/P buffer 1 | O
+// TMEM columns: Q (bf16 pairs) | S buffer 0 | S buffer 1 | O | P (bf16 pairs)
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t TQ = 0, TS = 64, TO = TS + 2 * 128;
-static_assert(TO + 128 <= TMEM_COLS, "TMEM budget");
+constexpr uint32_t TQ = 0, TS = 64, TO = TS + 2 * 128, TP = TO + 128;
+static_assert(TP + 64 <= TMEM_COLS, "TMEM budget");
 
 constexpr int NSOFT = NWG * 128;   // softmax threads
-constexpr int NTHREADS = NSOFT + 64;
-constexpr int W_TMA = NSOFT / 32, W_MMA = NSOFT / 32 + 1;
+constexpr int NTHREADS = NSOFT + 96;
+constexpr int W_TMA = NSOFT / 32, W_MMA = NSOFT / 32 + 1, W_TMA_V = NSOFT / 32 + 2;
 __device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory"); }
 
 struct Maps {
@@ -147,8 +147,13 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(B_SFULL + s), 1);
-            mbar_init(bar(B_PFULL + s), 8);         // one arrival per warp of the two groups
+            mbar_init(bar(B_SFREE + s), 8);         // one arrival per warp of the two groups
+            mbar_init(bar(B_PFULL + s), 8);
         }
+        // PV(t) commits to PFREE[t & 1]: each waiter then sees every phase of the barrier it waits on
+        // (a thread that skipped a phase could not tell it from the one two before)
+        mbar_init(bar(B_PFREE), 1);
+        mbar_init(bar(B_PFREE + 1), 1);
         mbar_init(bar(B_OFULL), 1);
         // rendezvous of the softmax threads after the first bounded wait: mbarriers, so that they
         // too can give up (a bar.sync would hang if one thread had left its loop)
@@ -234,10 +239,12 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const int T = (nU + 1) >> 1;   // 128-key tiles
 
     if (warp == W_TMA) {
-        // ================= TMA producer (whole warp in the loop, one elected lane issues) ======
+        // ===== K producer (whole warp in the loop, one elected lane issues) =====================
+        // K and V have a producer warp each: a K stage comes back as soon as S is computed, long
+        // before the V stage of the same tile does, and must not queue behind it.
         for (int t = 0; t < T; ++t) {
-            const int s = t % KSTAGES, sv = t % VSTAGES;
-            const uint32_t ph = (t / KSTAGES) & 1, phv = (t / VSTAGES) & 1;
+            const int s = t % KSTAGES;
+            const uint32_t ph = (t / KSTAGES) & 1;
             const int J0 = s_list[2 * t] >> 2;
             const int J1 = (2 * t + 1 < nU) ? (s_list[2 * t + 1] >> 2) : J0;  // odd tail: finite filler, masked
             if (!mbar_wait(bar(B_KEMPTY + s), ph ^ 1, s_abort, a.status, 0x1)) break;
@@ -250,6 +257,14 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 tma_load_4d(kd + 24576, &maps.k, bar(B_KFULL + s), 64, J1 * USV_BLOCK, h, b);
             }
             __syncwarp();
+        }
+    } else if (warp == W_TMA_V) {
+        // ===== V producer =======================================================================
+        for (int t = 0; t < T; ++t) {
+            const int sv = t % VSTAGES;
+            const uint32_t phv = (t / VSTAGES) & 1;
+            const int J0 = s_list[2 * t] >> 2;
+            const int J1 = (2 * t + 1 < nU) ? (s_list[2 * t + 1] >> 2) : J0;
             if (!mbar_wait(bar(B_VEMPTY + sv), phv ^ 1, s_abort, a.status, 0x2)) break;
             const uint32_t vd = base + SM_V + sv * TILE_BYTES;
             if (elect_one()) {
@@ -262,7 +277,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
             __syncwarp();
         }
     } else if (warp == W_MMA) {
-        // ================= MMA issuer (whole warp in the loop, one elected lane issues) ========
+        // ===== MMA issuer (whole warp in the loop, one elected lane issues); TMEM owner =========
         if (T > 0) {
             constexpr uint32_t IDESC_S = instr_desc(128, KT, 0, 0);    // Q (TMEM) x K (K-major)
             constexpr uint32_t IDESC_O = instr_desc(128, D, 0, 1);     // P (TMEM) x V (MN-major)
@@ -270,13 +285,17 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
             const uint64_t vdesc0 = smem_desc(base + SM_V, 16384, 1024);
             bool ok = mbar_wait(bar(B_QFULL), 0, s_abort, a.status, 0x4);
             fence_after();
-            // S(t) -> buffer t & 1.  The MMA that last read P from that buffer, PV(t - 2), has been
-            // issued by the time S(t) is (see the loop), and MMAs execute in issue order.
-            auto issue_s = [&](int t, bool k_ready) -> bool {
+            // S(t) -> buffer t & 1, once the softmax threads of tile t - 2 have taken its logits out
+            auto issue_s = [&](int t, bool k_ready, bool s_free) -> bool {
                 const int s = t % KSTAGES;
                 const uint32_t ph = (t / KSTAGES) & 1;
                 const int sb = t & 1;
                 if (!k_ready && !mbar_wait(bar(B_KFULL + s), ph, s_abort, a.status, 0x8)) return false;
+                if (t >= 2) {
+                    if (!s_free && !mbar_wait(bar(B_SFREE + sb), ((t - 2) >> 1) & 1, s_abort, a.status, 0x10))
+                        return false;
+                    fence_after();
+                }
                 const uint64_t kdesc = kdesc0 + ((s * TILE_BYTES) >> 4);
                 const uint32_t d_s = tmem + TS + sb * 128;
                 if (elect_one()) {
@@ -288,30 +307,33 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 }
                 return true;
             };
-            if (ok) ok = issue_s(0, false);
+            if (ok) ok = issue_s(0, false, true);
+            if (ok && T > 1) ok = issue_s(1, false, true);
             for (int t = 0; ok && t < T; ++t) {
                 const int sv = t % VSTAGES;
                 const uint32_t phv = (t / VSTAGES) & 1;
                 const int sb = t & 1;
-                // poll the three barriers of this step together: their latencies overlap
-                const int t1 = t + 1;
-                const bool k_rdy = t1 < T && mbar_try(bar(B_KFULL + t1 % KSTAGES), (t1 / KSTAGES) & 1);
+                // poll the barriers of this step together: their latencies overlap
+                const int t2 = t + 2;
+                const bool k_rdy = t2 < T && mbar_try(bar(B_KFULL + t2 % KSTAGES), (t2 / KSTAGES) & 1);
+                const bool f_rdy = t2 < T && mbar_try(bar(B_SFREE + sb), (t >> 1) & 1);
                 const bool v_rdy = mbar_try(bar(B_VFULL + sv), phv);
                 const bool p_rdy = mbar_try(bar(B_PFULL + sb), (t >> 1) & 1);
-                if (t1 < T) {
-                    ok = issue_s(t1, k_rdy);   // early: the softmax of tile t + 1 overlaps PV(t)
+                if (t2 < T) {
+                    // S two tiles ahead, issued while P(t) is still being made: its buffer was read
+                    // out long before, and the softmax threads need it as early as possible
+                    ok = issue_s(t2, k_rdy, f_rdy);
                     if (!ok) break;
                 }
                 if (!v_rdy && !mbar_wait(bar(B_VFULL + sv), phv, s_abort, a.status, 0x20)) break;
                 if (!p_rdy && !mbar_wait(bar(B_PFULL + sb), (t >> 1) & 1, s_abort, a.status, 0x40)) break;
                 fence_after();
                 const uint64_t vdesc = vdesc0 + ((sv * TILE_BYTES) >> 4);
-                const uint32_t a_p = tmem + TS + sb * 128;
                 if (elect_one()) {
 #pragma unroll
                     for (int ks = 0; ks < KT / 16; ++ks)
-                        umma_ts(tmem + TO, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vdesc + ((ks * 2048) >> 4), IDESC_O,
-                                (t > 0 || ks > 0));
+                        umma_ts(tmem + TO, tmem + TP + ks * 8, vdesc + ((ks * 2048) >> 4), IDESC_O, (t > 0 || ks > 0));
+                    umma_commit(bar(B_PFREE + sb));
                     if (t == T - 1) umma_commit(bar(B_OFULL));
                 }
             }
@@ -333,6 +355,8 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
         const uint64_t c2 = pack_f32x2(c, c);
         bool ok = true;
         const uint32_t sbase = lane_base + TS + tp * 128 + hb * 64;
+        const uint32_t pbase = lane_base + TP + hb * 32;
+        const bool releaser = hb == 0 && (warp & 3) == 0 && lane == 0;   // hands stages back
         for (int t = tp; t < T; t += 2) {
             const int slot = 2 * t + hb;
             const int e = slot < nU ? s_list[slot] : 0;
@@ -340,24 +364,19 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
             const int nv = N - (e >> 2) * USV_BLOCK;   // keys of the block with index < N
             if (!mbar_wait(bar(B_SFULL + tp), (t >> 1) & 1, s_abort, a.status, 0x80)) { ok = false; break; }
             fence_after();
-            if (hb == 0 && (warp & 3) == 0 && lane == 0) {
-                // S(t) is complete, and so is every MMA issued before it: PV(t - 2) and older
-                mbar_arrive(bar(B_KEMPTY + t % KSTAGES));
-                if (t >= 2) mbar_arrive(bar(B_VEMPTY + (t - 2) % VSTAGES));
-            }
-            uint32_t s0[32], s1[32];
-            if (mine) {
-                tmem_ld32(sbase, s0);
-                tmem_ld32(sbase + 32, s1);
-            }
+            if (releaser) mbar_arrive(bar(B_KEMPTY + t % KSTAGES));   // S(t) is complete
             if (!have_ref && slot >= sref) {
                 if (slot == sref) {
+                    // one-off pass over this key block for the row maximum (the block is mine here)
+                    uint32_t m0[32], m1[32];
+                    tmem_ld32(sbase, m0);
+                    tmem_ld32(sbase + 32, m1);
                     tmem_wait_ld();
                     float mx = -INFINITY;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        if (j < nv) mx = fmaxf(mx, __uint_as_float(s0[j]));
-                        if (j + 32 < nv) mx = fmaxf(mx, __uint_as_float(s1[j]));
+                        if (j < nv) mx = fmaxf(mx, __uint_as_float(m0[j]));
+                        if (j + 32 < nv) mx = fmaxf(mx, __uint_as_float(m1[j]));
                     }
                     nref = mx == -INFINITY ? 0.f : -mx * c;
                     s_refv[r] = nref;
@@ -370,27 +389,38 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 nref2 = pack_f32x2(nref, nref);
                 have_ref = true;
             }
-            // P overwrites the first 32 of the 64 logit columns just read
-            uint32_t pk[16];
-            if (mine) {
-                tmem_wait_ld();
-                if (nv >= USV_BLOCK) {
-                    weights32<false>(s0, pk, c2, nref2, 0, nv, lr2);
-                    tmem_st16(sbase, pk);
-                    weights32<false>(s1, pk, c2, nref2, 32, nv, lr2);
-                    tmem_st16(sbase + 16, pk);
-                } else {
-                    weights32<true>(s0, pk, c2, nref2, 0, nv, lr2);
-                    tmem_st16(sbase, pk);
-                    weights32<true>(s1, pk, c2, nref2, 32, nv, lr2);
-                    tmem_st16(sbase + 16, pk);
+            // Half of the 64 logit columns at a time, to stay within the register budget; the S
+            // buffer is handed back as soon as the second half is in registers.
+            uint32_t pk0[16], pk1[16];
+            {
+                uint32_t sx[32];
+                if (mine) {
+                    tmem_ld32(sbase, sx);
+                    tmem_wait_ld();
+                    if (nv >= USV_BLOCK) weights32<false>(sx, pk0, c2, nref2, 0, nv, lr2);
+                    else weights32<true>(sx, pk0, c2, nref2, 0, nv, lr2);
+                    tmem_ld32(sbase + 32, sx);
                 }
-            } else {
+                tmem_wait_ld();
+                fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_SFREE + tp));
+                if (mine) {
+                    if (nv >= USV_BLOCK) weights32<false>(sx, pk1, c2, nref2, 32, nv, lr2);
+                    else weights32<true>(sx, pk1, c2, nref2, 32, nv, lr2);
+                } else {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) pk[j] = 0u;
-                tmem_st16(sbase, pk);
-                tmem_st16(sbase + 16, pk);
+                    for (int j = 0; j < 16; ++j) pk0[j] = pk1[j] = 0u;
+                }
             }
+            if (t > 0) {
+                // the P buffer is free once PV(t - 1) has read it; that also frees its V stage
+                if (!mbar_wait(bar(B_PFREE + (tp ^ 1)), ((t - 1) >> 1) & 1, s_abort, a.status, 0x100)) { ok = false; break; }
+                fence_after();
+                if (releaser) mbar_arrive(bar(B_VEMPTY + (t - 1) % VSTAGES));
+            }
+            tmem_st16(pbase, pk0);
+            tmem_st16(pbase + 16, pk1);
             tmem_wait_st();
             fence_before();
             __syncwarp();
