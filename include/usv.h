@@ -125,6 +125,13 @@ int usv_select_blocks(int B, int H, int NBq, int NBk, const float* scores,
  * lse: optional fp32 [B,H,N], natural-log of the softmax denominator (NULL to skip).
  * scale: logit scale; 0 selects 1/sqrt(d).
  * impl: 0 = default kernel, 1 = legacy mma.sync kernel (kept as an on-device cross-check).
+ *
+ * The default kernel (d = 128) computes two neighbouring query blocks together over the union of
+ * their key-block lists and gives a key block that only one of them selected zero weight for
+ * the other.  Results equal the per-block definition for finite inputs.  A NaN or infinity in K
+ * or V inside a block that one query block of a pair selected can also reach the output rows of
+ * its partner (0 * inf); blocks that neither selected are never read.  impl 1 keeps query blocks
+ * fully separate.
  */
 size_t usv_sparse_attn_workspace(int B, int H, int N, int d, int kmax);
 int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,

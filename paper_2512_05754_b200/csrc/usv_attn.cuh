@@ -25,8 +25,6 @@ struct AttnArgs {
 };
 
 int launch_attn_mma(const AttnArgs& a, int d, cudaStream_t st);
-bool attn_tc_supported(const AttnArgs& a, int d);
-int launch_attn_tc(const AttnArgs& a, int d, cudaStream_t st);
 bool attn_pair_supported(const AttnArgs& a, int d);
 int launch_attn_pair(const AttnArgs& a, int d, cudaStream_t st);
 

@@ -28,7 +28,7 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     if (sel == nullptr || k_per_head == nullptr) return fail(USV_ERR_INVALID_ARG, "sparse_attn: null sel/k_per_head");
     if (o_f32 != nullptr && !aligned16(o_f32)) return fail(USV_ERR_UNSUPPORTED, "sparse_attn: o_f32 misaligned");
     if (!(scale >= 0.f)) return fail(USV_ERR_INVALID_ARG, "sparse_attn: scale must be >= 0");
-    if (impl < 0 || impl > 2) return fail(USV_ERR_INVALID_ARG, "sparse_attn: impl must be 0, 1 or 2");
+    if (impl != 0 && impl != 1) return fail(USV_ERR_INVALID_ARG, "sparse_attn: impl must be 0 or 1");
     if (ws == nullptr) return fail(USV_ERR_INVALID_ARG, "sparse_attn: null workspace");
     if (ws_bytes < usv_sparse_attn_workspace(B, H, N, d, kmax))
         return fail(USV_ERR_WORKSPACE, "sparse_attn: workspace %zu < %zu", ws_bytes,
@@ -66,9 +66,8 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemsetAsync(ws, 0, 256, st);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: memset: %s", cudaGetErrorString(e));
-    const bool pair_ok = impl == 0 && attn_pair_supported(a, d);
-    if (pair_ok || (impl != 1 && attn_tc_supported(a, d))) {
-        int rc2 = pair_ok ? launch_attn_pair(a, d, st) : launch_attn_tc(a, d, st);
+    if (impl == 0 && attn_pair_supported(a, d)) {
+        int rc2 = launch_attn_pair(a, d, st);
         if (rc2 != USV_OK) return rc2;
         // exact recomputation of the (normally zero) query blocks the fast kernel reported
         a.work_list = a.fallback_list;
