@@ -4,6 +4,8 @@
 
 namespace usv {
 
+constexpr int PLAN_WINDOW = 64;   // pairing looks at this many query blocks on each side
+
 struct AttnArgs {
     const __nv_bfloat16 *q, *k, *v;
     __nv_bfloat16* o;
@@ -16,6 +18,7 @@ struct AttnArgs {
     // their work ids here; the exact kernel, launched in list mode, recomputes them.
     int* fallback_list;
     int* fallback_count;
+    const int2* pairs;      // [B,H,ceil(NB/2)] query-block pairs of the tcgen05 kernel (head-major, not head-ordered)
     const int* work_list;   // list mode of the exact kernel (NULL = one CTA per query block)
     const int* work_count;
     int B, H, N, NB, kmax;
@@ -27,5 +30,7 @@ struct AttnArgs {
 int launch_attn_mma(const AttnArgs& a, int d, cudaStream_t st);
 bool attn_pair_supported(const AttnArgs& a, int d);
 int launch_attn_pair(const AttnArgs& a, int d, cudaStream_t st);
+size_t pair_plan_bytes(int B, int H, int NB);
+int launch_pair_plan(const AttnArgs& a, void* mem, cudaStream_t st);
 
 }  // namespace usv

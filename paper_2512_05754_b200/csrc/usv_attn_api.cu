@@ -6,8 +6,9 @@
 extern "C" size_t usv_sparse_attn_workspace(int B, int H, int N, int d, int kmax) {
     (void)d; (void)kmax;
     if (B <= 0 || H <= 0 || N <= 0) return 0;
-    // status word + fallback counter (256-byte header), then the fallback work list
-    return 256 + usv::align_up((size_t)B * H * usv::ceil_div(N, USV_BLOCK) * sizeof(int), 256);
+    // status word + fallback counter (256-byte header), the fallback work list, the pairing plan
+    const int NB = usv::ceil_div(N, USV_BLOCK);
+    return 256 + usv::align_up((size_t)B * H * NB * sizeof(int), 256) + usv::pair_plan_bytes(B, H, NB);
 }
 
 extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,
@@ -58,6 +59,8 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     a.status = static_cast<unsigned int*>(ws);
     a.fallback_count = reinterpret_cast<int*>(static_cast<char*>(ws) + 4);
     a.fallback_list = reinterpret_cast<int*>(static_cast<char*>(ws) + 256);
+    void* plan_mem = static_cast<char*>(ws) + 256 + align_up((size_t)B * H * NB * sizeof(int), 256);
+    a.pairs = static_cast<const int2*>(plan_mem);
     a.work_list = nullptr;
     a.work_count = nullptr;
     a.B = B; a.H = H; a.N = N; a.NB = NB; a.kmax = kmax;
@@ -67,7 +70,9 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     cudaError_t e = cudaMemsetAsync(ws, 0, 256, st);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: memset: %s", cudaGetErrorString(e));
     if (impl == 0 && attn_pair_supported(a, d)) {
-        int rc2 = launch_attn_pair(a, d, st);
+        int rc2 = launch_pair_plan(a, plan_mem, st);
+        if (rc2 != USV_OK) return rc2;
+        rc2 = launch_attn_pair(a, d, st);
         if (rc2 != USV_OK) return rc2;
         // exact recomputation of the (normally zero) query blocks the fast kernel reported
         a.work_list = a.fallback_list;

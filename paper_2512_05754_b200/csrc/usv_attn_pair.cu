@@ -10,8 +10,9 @@
 //
 // A key block that only one of the two lists holds is masked for the other half of the rows
 // (its softmax weights are written as zero), so the result is exactly the per-block selection.
-// Neighbouring query blocks of video tokens select largely the same key blocks, which is what
-// makes the shared tile pay.
+// Nearby query blocks of video tokens select largely the same key blocks, which is what makes
+// the shared tile pay; which two blocks share a CTA is chosen per call for large list overlap
+// (usv_attn_plan.cu).
 //
 // Query rows live on TMEM lanes: softmax thread i owns row i, so maxima and sums need no
 // cross-thread traffic.  The softmax reference of a row (the value subtracted inside the
@@ -122,8 +123,9 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const int b = bh_ord / a.H;
     const int h = a.head_order[bh_ord % a.H];
     const int kh = a.k_per_head[h];
-    const int IA = 2 * pair;
-    const int IB = (2 * pair + 1 < NB) ? 2 * pair + 1 : -1;
+    const int2 pq = a.pairs[((int64_t)b * a.H + h) * NP + pair];   // similarity-driven pairing
+    const int IA = pq.x;
+    const int IB = pq.y;
     const int nwords = (NB + 31) >> 5;
 
     // softmax-thread geometry (meaningful for warps < W_TMA)
@@ -197,7 +199,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
             if (J >= 0 && J < NB) atomicOr(&bitsA[J >> 5], 1u << (J & 31));
         }
         if (IB >= 0) {
-            const int32_t* selB = selA + a.kmax;
+            const int32_t* selB = a.sel + (((int64_t)b * a.H + h) * NB + IB) * a.kmax;
             for (int t = tid; t < kh; t += NSOFT) {
                 const int J = selB[t];
                 if (J >= 0 && J < NB) atomicOr(&bitsB[J >> 5], 1u << (J & 31));
