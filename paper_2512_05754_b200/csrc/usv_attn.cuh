@@ -19,6 +19,11 @@ struct AttnArgs {
     int* fallback_list;
     int* fallback_count;
     const int2* pairs;      // [B,H,ceil(NB/2)] query-block pairs of the tcgen05 kernel (head-major, not head-ordered)
+    // Union key-block lists of the pairs: for (b, h, pair) at lists + b * list_batch + list_off[h] +
+    // pair * list_stride(h): [0] = number of entries, then (key block << 2) | in-A | in-B << 1, ascending.
+    const int* lists;
+    int64_t list_batch;
+    int64_t list_off[USV_MAX_HEADS];
     const int* work_list;   // list mode of the exact kernel (NULL = one CTA per query block)
     const int* work_count;
     int B, H, N, NB, kmax;
@@ -30,7 +35,10 @@ struct AttnArgs {
 int launch_attn_mma(const AttnArgs& a, int d, cudaStream_t st);
 bool attn_pair_supported(const AttnArgs& a, int d);
 int launch_attn_pair(const AttnArgs& a, int d, cudaStream_t st);
-size_t pair_plan_bytes(int B, int H, int NB);
-int launch_pair_plan(const AttnArgs& a, void* mem, cudaStream_t st);
+// ints one pair's list occupies for a head that keeps k of NB key blocks (header + entries)
+__host__ __device__ inline int64_t list_stride(int k, int NB) { return 1 + (int64_t)(2 * (int64_t)k < NB ? 2 * k : NB); }
+size_t pair_plan_bytes(int B, int H, int NB, const int32_t* k_per_head);
+// Fills a.pairs / a.lists / a.list_* (pointing into mem) and enqueues the plan kernels.
+int launch_pair_plan(AttnArgs& a, void* mem, cudaStream_t st);
 
 }  // namespace usv

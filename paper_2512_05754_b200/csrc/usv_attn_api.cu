@@ -4,11 +4,15 @@
 #include "usv_attn.cuh"
 
 extern "C" size_t usv_sparse_attn_workspace(int B, int H, int N, int d, int kmax) {
-    (void)d; (void)kmax;
+    (void)d;
     if (B <= 0 || H <= 0 || N <= 0) return 0;
     // status word + fallback counter (256-byte header), the fallback work list, the pairing plan
     const int NB = usv::ceil_div(N, USV_BLOCK);
-    return 256 + usv::align_up((size_t)B * H * NB * sizeof(int), 256) + usv::pair_plan_bytes(B, H, NB);
+    // sized for the worst case of every head keeping kmax blocks
+    if (H > USV_MAX_HEADS) return 0;
+    int32_t kk[USV_MAX_HEADS];
+    for (int h = 0; h < H; ++h) kk[h] = kmax < 1 ? 1 : (kmax > NB ? NB : kmax);
+    return 256 + usv::align_up((size_t)B * H * NB * sizeof(int), 256) + usv::pair_plan_bytes(B, H, NB, kk);
 }
 
 extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,
@@ -60,7 +64,9 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     a.fallback_count = reinterpret_cast<int*>(static_cast<char*>(ws) + 4);
     a.fallback_list = reinterpret_cast<int*>(static_cast<char*>(ws) + 256);
     void* plan_mem = static_cast<char*>(ws) + 256 + align_up((size_t)B * H * NB * sizeof(int), 256);
-    a.pairs = static_cast<const int2*>(plan_mem);
+    a.pairs = nullptr;
+    a.lists = nullptr;
+    a.list_batch = 0;
     a.work_list = nullptr;
     a.work_count = nullptr;
     a.B = B; a.H = H; a.N = N; a.NB = NB; a.kmax = kmax;

@@ -58,8 +58,7 @@ enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = B_KFULL + KSTAGES, B_VFULL = B_KEMPT
        B_PFULL = B_SFREE + 2, B_PFREE = B_PFULL + 2, B_OFULL = B_PFREE + 2, B_REF, B_EPI = B_REF + 2, B_COUNT = B_EPI + 2 };
 static_assert(B_COUNT <= 32, "barrier area");
 constexpr uint32_t SM_MISC = SM_BAR + 8 * 32;            // tmem base, abort flag, flags, union size
-constexpr uint32_t SM_BITS = SM_MISC + 64;               // two bitmaps of MAX_NB bits
-constexpr uint32_t SM_LIST = SM_BITS + 2 * (MAX_NB / 8); // int[MAX_NB]: (key block << 2) | in-A | in-B << 1
+constexpr uint32_t SM_LIST = SM_MISC + 64;               // int[MAX_NB]: (key block << 2) | in-A | in-B << 1
 constexpr uint32_t SM_REFV = SM_LIST + MAX_NB * 4;       // float[128]: minus the softmax reference per row
 constexpr uint32_t SM_SUM = SM_REFV + 128 * 4;           // float[NWG][128]: partial row sums
 constexpr uint32_t SM_TOTAL = SM_SUM + NWG * 128 * 4;
@@ -110,7 +109,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     volatile int* s_abort = reinterpret_cast<volatile int*>(sm + SM_MISC + 4);
     volatile int* s_flag = reinterpret_cast<volatile int*>(sm + SM_MISC + 8);   // [2]
     volatile int* s_nu = reinterpret_cast<volatile int*>(sm + SM_MISC + 16);
-    uint32_t* s_bits = reinterpret_cast<uint32_t*>(sm + SM_BITS);
     int* s_list = reinterpret_cast<int*>(sm + SM_LIST);
     float* s_refv = reinterpret_cast<float*>(sm + SM_REFV);
     float* s_sum = reinterpret_cast<float*>(sm + SM_SUM);
@@ -126,7 +124,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const int2 pq = a.pairs[((int64_t)b * a.H + h) * NP + pair];   // similarity-driven pairing
     const int IA = pq.x;
     const int IB = pq.y;
-    const int nwords = (NB + 31) >> 5;
 
     // softmax-thread geometry (meaningful for warps < W_TMA)
     const int grp = warp >> 2;                       // tiles of parity grp >> 1, key block grp & 1
@@ -136,7 +133,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const int row = Iq * USV_BLOCK + (r & 63);
     const bool live = Iq >= 0 && row < N;
 
-    // ---- set-up: barriers, TMEM, ascending union of the two selection rows, Q -> TMEM
+    // ---- set-up: barriers, TMEM, the pair's key-block list -> shared memory, Q -> TMEM
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), NSOFT / 32);       // one arrival per softmax warp
         for (int s = 0; s < KSTAGES; ++s) {
@@ -173,17 +170,18 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                      ::"r"(base + SM_MISC), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    uint32_t* bitsA = s_bits;
-    uint32_t* bitsB = s_bits + MAX_NB / 32;
+    const int* plist = a.lists + b * a.list_batch + a.list_off[h] + (int64_t)pair * list_stride(kh, NB);
     uint4 qv[4];   // this thread's quarter of its query row (32 of the 128 bf16)
     if (warp < W_TMA) {
         const uint4* src = reinterpret_cast<const uint4*>(a.q + b * a.sq.sb + h * a.sq.sh +
                                                           (int64_t)row * a.sq.sn + grp * 32);
 #pragma unroll
         for (int i = 0; i < 4; ++i) qv[i] = live ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
-        for (int w = threadIdx.x; w < nwords; w += NSOFT) {
-            bitsA[w] = 0;
-            bitsB[w] = 0;
+        // the pair's union key-block list (built by the plan kernels) -> shared memory
+        const int lstride = (int)list_stride(kh, NB);
+        for (int i = threadIdx.x; i < lstride; i += NSOFT) {
+            const int e = plist[i];
+            if (i == 0) *s_nu = e; else s_list[i - 1] = e;
         }
     }
     fence_before();
@@ -192,19 +190,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const uint32_t tmem = *s_tmem;
     const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     if (warp < W_TMA) {
-        const int tid = threadIdx.x;
-        const int32_t* selA = a.sel + (((int64_t)b * a.H + h) * NB + IA) * a.kmax;
-        for (int t = tid; t < kh; t += NSOFT) {
-            const int J = selA[t];
-            if (J >= 0 && J < NB) atomicOr(&bitsA[J >> 5], 1u << (J & 31));
-        }
-        if (IB >= 0) {
-            const int32_t* selB = a.sel + (((int64_t)b * a.H + h) * NB + IB) * a.kmax;
-            for (int t = tid; t < kh; t += NSOFT) {
-                const int J = selB[t];
-                if (J >= 0 && J < NB) atomicOr(&bitsB[J >> 5], 1u << (J & 31));
-            }
-        }
         // this thread's part of its query row -> TMEM (two bf16 of consecutive d per column)
         uint32_t q[16];
 #pragma unroll
@@ -216,27 +201,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
         fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(B_QFULL));
-        softmax_bar();
-        if (warp == 0) {
-            int running = 0;
-            for (int w0 = 0; w0 < nwords; w0 += 32) {
-                const int w = w0 + lane;
-                const uint32_t ba = w < nwords ? bitsA[w] : 0u;
-                const uint32_t bb = w < nwords ? bitsB[w] : 0u;
-                uint32_t u = ba | bb;
-                const int incl = warp_incl_scan(__popc(u));
-                int off = running + incl - __popc(u);
-                while (u) {
-                    const int bit = __ffs(u) - 1;
-                    u &= u - 1;
-                    s_list[off++] = ((w * 32 + bit) << 2) | ((ba >> bit) & 1u) | (((bb >> bit) & 1u) << 1);
-                }
-                running += __shfl_sync(0xffffffffu, incl, 31);
-            }
-            if (lane == 0) *s_nu = running;
-        }
     }
-    __syncthreads();
     const int nU = *s_nu;
     const int T = (nU + 1) >> 1;   // 128-key tiles
 
