@@ -45,7 +45,7 @@ using namespace t5;
 constexpr int D = 128;
 constexpr int KT = 2 * USV_BLOCK;               // keys per tile = two key blocks
 constexpr int NWG = 4;                          // softmax warpgroups
-constexpr int KSTAGES = 3;                      // K tile stages
+constexpr int KSTAGES = 2;                      // K tile stages
 constexpr int VSTAGES = 3;                      // V tile stages
 constexpr int MAX_NB = 4096;                    // key blocks per sequence this kernel covers
 constexpr uint32_t TILE_BYTES = KT * D * 2;     // 32 KB: [d-half][128 keys][128 B]
