@@ -384,7 +384,9 @@ __global__ void __launch_bounds__(256) merge_kernel(Part p, int N, int C, int nU
         return;
     }
     int myid = 0x7fffffff;
-    if (len <= 32) {
+    if (len == 1) {
+        myid = list[0];
+    } else if (len <= 32) {
         // rank sort in registers: lane s ends up holding the s-th smallest source index
         const int id = lane < len ? list[lane] : 0x7fffffff;
         int rank = 0;
@@ -423,24 +425,43 @@ __global__ void __launch_bounds__(256) merge_kernel(Part p, int N, int C, int nU
         }
     }
     const float inv = 1.0f / (float)(len + 1);
-    for (int c0 = 0; c0 < nvec; c0 += 32) {
-        const int c = c0 + lane;
-        const bool act = c < nvec;
-        float acc[8];
-        if (act) bf16x8_to_float(__ldg(srcj + c), acc);
+    // G 16-byte chunks per lane at a time: the loads of one row are all in flight together, and
+    // rows are added in ascending source index (fp32)
+    constexpr int G = 3;
+    for (int c0 = 0; c0 < nvec; c0 += 32 * G) {
+        float acc[G][8];
+        uint4 v[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const int c = c0 + g * 32 + lane;
+            v[g] = c < nvec ? __ldg(srcj + c) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) bf16x8_to_float(v[g], acc[g]);
         for (int s = 0; s < len; ++s) {
             const int i = len <= 32 ? __shfl_sync(0xffffffffu, myid, s) : list[s];
-            if (act) {
-                float f[8];
-                bf16x8_to_float(__ldg(reinterpret_cast<const uint4*>(xb + (int64_t)i * C) + c), f);
+            const uint4* srci = reinterpret_cast<const uint4*>(xb + (int64_t)i * C);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] += f[e];
+            for (int g = 0; g < G; ++g) {
+                const int c = c0 + g * 32 + lane;
+                v[g] = c < nvec ? __ldg(srci + c) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float f[8];
+                bf16x8_to_float(v[g], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g][e] += f[e];
             }
         }
-        if (act) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] *= inv;
-            dst[c] = float8_to_bf16x8(acc);
+        for (int g = 0; g < G; ++g) {
+            const int c = c0 + g * 32 + lane;
+            if (c < nvec) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g][e] *= inv;
+                dst[c] = float8_to_bf16x8(acc[g]);
+            }
         }
     }
 }
