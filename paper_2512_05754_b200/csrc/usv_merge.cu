@@ -12,27 +12,9 @@
 //   unmerge_kernel     Eq. 15    warp-per-row gather copy, 16-byte accesses
 #include <math.h>
 
-#include "usv_common.cuh"
+#include "usv_match.cuh"
 
 namespace usv {
-
-struct Part {
-    int T, Hh, W, st, sh, sw;
-    int nHy, nWx, nB;  // destinations per axis (y, x) and in total
-    __host__ __device__ bool is_dst(int n) const {
-        const int x = n % W, y = (n / W) % Hh, t = n / (W * Hh);
-        return (t % st == 0) && (y % sh == 0) && (x % sw == 0);
-    }
-    // ordinal (ascending token order) of a destination token
-    __host__ __device__ int ord(int n) const {
-        const int x = n % W, y = (n / W) % Hh, t = n / (W * Hh);
-        return ((t / st) * nHy + y / sh) * nWx + x / sw;
-    }
-    __host__ __device__ int dst_token(int o) const {
-        const int dx = o % nWx, dy = (o / nWx) % nHy, dt = o / (nWx * nHy);
-        return ((dt * st) * Hh + dy * sh) * W + dx * sw;
-    }
-};
 
 // ---------------------------------------------------------------------------- descriptors
 // One warp per token.  DM/8 lanes cover one head's row with 16-byte loads; 32/(DM/8) heads are
@@ -484,7 +466,7 @@ __global__ void __launch_bounds__(256) unmerge_kernel(int N, int Nm, int C,
 
 // ---------------------------------------------------------------------------- host side
 struct MergeWs {
-    size_t mhat, src_idx, jstar_s, u_s, row_src, cnt, off, cursor, csr, total;
+    size_t mhat, src_idx, jstar_s, u_s, row_src, cnt, off, cursor, csr, status, split, total;
 };
 
 static MergeWs merge_layout(int B, int N, int dm, int nA, int nB) {
@@ -500,6 +482,8 @@ static MergeWs merge_layout(int B, int N, int dm, int nA, int nB) {
     w.off = take((size_t)B * (nB + 1) * 4);
     w.cursor = take((size_t)B * nB * 4);
     w.csr = take((size_t)B * nA * 4);
+    w.status = take(256);                                       // device status word of the bounded waits
+    w.split = take(dm == 128 ? match_tc_bytes(B, N) : 0);       // bf16 hi/lo planes of the tensor-core matcher
     w.total = o;
     return w;
 }
@@ -565,10 +549,18 @@ extern "C" int usv_token_merge(int B, int N, int C, const void* x, int Hm, int d
         if (nA > 0) {
             src_list_kernel<<<1, 1024, 0, s>>>(p, N, src_idx);
             USV_CHECK_LAUNCH("src_list_kernel");
-            dim3 mg(ceil_div(nA, 64), B);
-            if (dm == 128) match_kernel<128><<<mg, 256, 0, s>>>(mhat, p, N, nA, src_idx, jstar_s, u_s);
-            else match_kernel<64><<<mg, 256, 0, s>>>(mhat, p, N, nA, src_idx, jstar_s, u_s);
-            USV_CHECK_LAUNCH("match_kernel");
+            if (dm == 128) {
+                // tensor cores: split-bf16 cosines (usv_match_tc.cu)
+                unsigned int* status = reinterpret_cast<unsigned int*>(base + L.status);
+                cudaError_t e0 = cudaMemsetAsync(status, 0, 4, s);
+                if (e0 != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: memset: %s", cudaGetErrorString(e0));
+                int rc = launch_match_tc(mhat, p, B, N, nA, src_idx, jstar_s, u_s, base + L.split, status, s);
+                if (rc != USV_OK) return rc;
+            } else {
+                dim3 mg(ceil_div(nA, 64), B);
+                match_kernel<64><<<mg, 256, 0, s>>>(mhat, p, N, nA, src_idx, jstar_s, u_s);
+                USV_CHECK_LAUNCH("match_kernel");
+            }
         }
         plan_kernel<<<B, 1024, 0, s>>>(p, N, nA, r, src_idx, jstar_s, u_s, dst_of, pos, u_out, jstar_out);
         USV_CHECK_LAUNCH("plan_kernel");
