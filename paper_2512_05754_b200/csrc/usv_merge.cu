@@ -77,18 +77,19 @@ __device__ __forceinline__ int block_scan_1024(int v, int* scratch, int* total) 
     return res;
 }
 
-// Ascending list of the source tokens (same for every batch element).  One CTA, 1024 threads.
-__global__ void __launch_bounds__(1024) src_list_kernel(Part p, int N, int32_t* __restrict__ src_idx) {
-    __shared__ int scratch[33];
-    int base = 0;
-    for (int n0 = 0; n0 < N; n0 += 1024) {
-        const int n = n0 + threadIdx.x;
-        const int flag = (n < N && !p.is_dst(n)) ? 1 : 0;
-        int tot;
-        const int r = base + block_scan_1024(flag, scratch, &tot);
-        if (flag) src_idx[r] = n;
-        base += tot;
+// Ascending list of the source tokens (same for every batch element): the rank of a source is
+// its token index minus the number of destinations before it, which the partition gives in
+// closed form, so every token is handled independently.
+__global__ void __launch_bounds__(256) src_list_kernel(Part p, int N, int32_t* __restrict__ src_idx) {
+    const int n = blockIdx.x * 256 + threadIdx.x;
+    if (n >= N || p.is_dst(n)) return;
+    const int x = n % p.W, y = (n / p.W) % p.Hh, t = n / (p.W * p.Hh);
+    int before = ((t + p.st - 1) / p.st) * p.nHy * p.nWx;      // whole destination frames before t
+    if (t % p.st == 0) {
+        before += ((y + p.sh - 1) / p.sh) * p.nWx;              // whole destination rows before y
+        if (y % p.sh == 0) before += (x + p.sw - 1) / p.sw;     // destinations before x in this row
     }
+    src_idx[n - before] = n;
 }
 
 // ---------------------------------------------------------------------------- matching
@@ -547,7 +548,7 @@ extern "C" int usv_token_merge(int B, int N, int C, const void* x, int Hm, int d
         else desc_kernel<64><<<dg, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(metric), mhat, tokens, Hm);
         USV_CHECK_LAUNCH("desc_kernel");
         if (nA > 0) {
-            src_list_kernel<<<1, 1024, 0, s>>>(p, N, src_idx);
+            src_list_kernel<<<ceil_div(N, 256), 256, 0, s>>>(p, N, src_idx);
             USV_CHECK_LAUNCH("src_list_kernel");
             if (dm == 128) {
                 // tensor cores: split-bf16 cosines (usv_match_tc.cu)
