@@ -1,4 +1,11 @@
-// Top-k key-block selection: one CTA per score row.
+// Top-k key-block selection.
+//
+// Rows of up to 2048 scores (every workload here): one WARP per row, select_warp_kernel.  Each
+// lane keeps a contiguous chunk of the row as order-preserving keys in registers; the key T of
+// the k-th largest element is found bit by bit (32 warp-wide counts), then the lanes emit, in
+// ascending index, every element above T and the first (k - above) elements equal to T.
+//
+// Longer rows: one CTA per row, select_kernel.
 //
 // The row is mapped to order-preserving 32-bit keys in shared memory.  Four 8-bit radix passes
 // (most significant digit first) find the key T of the k-th largest element and the number of
@@ -114,6 +121,55 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* __rest
     for (int t = k + threadIdx.x; t < kmax; t += SEL_THREADS) out[t] = -1;
 }
 
+// One warp per row; lane l holds indices [l * KPL, (l + 1) * KPL).
+template <int KPL>
+__global__ void __launch_bounds__(256) select_warp_kernel(const float* __restrict__ scores,
+                                                          int32_t* __restrict__ sel, int H, int NBq,
+                                                          int NBk, int kmax, const SelHeads heads,
+                                                          int64_t rows) {
+    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int lane = threadIdx.x & 31;
+    const int h = (int)((row / NBq) % H);
+    const int k = heads.k[h];
+    const float* src = scores + row * NBk;
+    int32_t* out = sel + row * kmax;
+    const int j0 = lane * KPL;
+    uint32_t key[KPL];
+#pragma unroll
+    for (int i = 0; i < KPL; ++i) key[i] = (j0 + i < NBk) ? float_key(__ldg(src + j0 + i)) : 0u;   // 0 < any real key
+    // largest T with count(key >= T) >= k, one bit at a time
+    uint32_t T = 0;
+#pragma unroll 1
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t cand = T | (1u << bit);
+        int c = 0;
+#pragma unroll
+        for (int i = 0; i < KPL; ++i) c += key[i] >= cand ? 1 : 0;
+        if (__reduce_add_sync(0xffffffffu, c) >= k) T = cand;
+    }
+    int ngt = 0, neq = 0;
+#pragma unroll
+    for (int i = 0; i < KPL; ++i) {
+        ngt += key[i] > T ? 1 : 0;
+        neq += (key[i] == T && j0 + i < NBk) ? 1 : 0;
+    }
+    const int need_eq = k - __reduce_add_sync(0xffffffffu, ngt);   // kept among the equal ones: lowest indices
+    const int eq_before = warp_incl_scan(neq) - neq;
+    const int eq_take = min(max(need_eq - eq_before, 0), neq);
+    const int ntake = ngt + eq_take;
+    int p = warp_incl_scan(ntake) - ntake;
+    int eq_left = eq_take;
+#pragma unroll
+    for (int i = 0; i < KPL; ++i) {
+        const bool gt = key[i] > T;
+        const bool eq = key[i] == T && j0 + i < NBk && eq_left > 0;
+        if (gt || eq) out[p++] = j0 + i;
+        if (eq) --eq_left;
+    }
+    for (int t = k + lane; t < kmax; t += 32) out[t] = -1;
+}
+
 }  // namespace usv
 
 extern "C" int usv_select_blocks(int B, int H, int NBq, int NBk, const float* scores,
@@ -137,8 +193,13 @@ extern "C" int usv_select_blocks(int B, int H, int NBq, int NBk, const float* sc
     if (kmax < kmx) return fail(USV_ERR_INVALID_ARG, "select_blocks: kmax=%d < max k=%d", kmax, kmx);
     const int64_t rows = (int64_t)B * H * NBq;
     if (rows > 2147483647LL) return fail(USV_ERR_UNSUPPORTED, "select_blocks: too many rows");
-    select_kernel<<<(unsigned)rows, SEL_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
-        scores, sel, H, NBq, NBk, kmax, heads);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const unsigned wg = (unsigned)((rows + 7) / 8);
+    if (NBk <= 512) select_warp_kernel<16><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows);
+    else if (NBk <= 1024) select_warp_kernel<32><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows);
+    else if (NBk <= 1536) select_warp_kernel<48><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows);
+    else if (NBk <= 2048) select_warp_kernel<64><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows);
+    else select_kernel<<<(unsigned)rows, SEL_THREADS, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads);
     USV_CHECK_LAUNCH("select_kernel");
     return USV_OK;
 }

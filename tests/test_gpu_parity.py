@@ -117,7 +117,9 @@ def test_keep_all_matches_dense_attention(usv):
 def test_select_kernel_exact_on_tied_scores(usv):
     """Integer-valued scores with many exact ties: the tie rule must hold bit-exactly."""
     g = torch.Generator().manual_seed(11)
-    for NBk, ks in ((16, [1, 16, 5]), (300, [7, 150, 299]), (1393, [70, 349, 1393])):
+    # rows up to 2048 scores take the warp-per-row kernel, longer ones the CTA-per-row kernel
+    for NBk, ks in ((16, [1, 16, 5]), (300, [7, 150, 299]), (1393, [70, 349, 1393]), (2048, [1, 2048, 777]),
+                    (2500, [3, 1250, 2500])):
         s = torch.randint(-3, 4, (2, 3, 9, NBk), generator=g).float()
         s[0, 0, 0] = 0.0
         s[1, 2, 3] = -0.0
