@@ -111,6 +111,20 @@ def flops(wl, N, k_per_head):
     return dense, eff
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of per-rank timings over all ranks (every rank gets the result).
+    The job is as slow as its slowest rank; there is no data-path collective besides this."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_value(world, flops_per_rank, ms_per_step):
+    """Whole-job throughput in TFLOP/s: every rank runs one layer instance (weak scaling)."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 def build_inputs(wl, device):
     """Device-resident inputs of one step.  Returns a dict."""
     if wl.merge_part is None:
@@ -215,10 +229,7 @@ def run_usv(args, wl, rank, world, device):
     barrier()
     e2e_ms = f0.elapsed_time(f1) / e2e_steps
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=device)
-    if world > 1:
-        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
-    total_ms, e2e_ms = times.tolist()
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, device)
     if rank != 0:
         return None
     ms_step = total_ms / args.steps
@@ -230,7 +241,7 @@ def run_usv(args, wl, rank, world, device):
     pool_bytes = 2 * (wl.B * wl.H * N * wl.d * 2) + 2 * (wl.B * wl.H * ((N + 63) // 64) * wl.d * 4)
     result = {
         "metric": "sparse_attn_dense_equiv_tflops",
-        "value": world * dense_f / (ms_step * 1e-3) / 1e12,
+        "value": job_value(world, dense_f, ms_step),
         "unit": "TFLOP/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step,
@@ -258,7 +269,7 @@ def run_usv(args, wl, rank, world, device):
                      "achieved": attn_eff_tflops, "peak": peak, "unit": "TFLOP/s",
                      "frac": attn_eff_tflops / peak, "peak_source": "%s (burst bf16)" % peak_src,
                      "traffic": ATTN_DRAM_TRAFFIC.get(wl.name)},
-        "e2e": {"value": world * dense_f / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+        "e2e": {"value": job_value(world, dense_f, e2e_ms), "unit": "TFLOP/s",
                 "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(3 * hq.numel() * 2), "d2h_bytes_per_step": int(ho.numel() * 2)},
         "gpu_launches": launches_per_step * args.steps,
