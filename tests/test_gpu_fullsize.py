@@ -69,6 +69,15 @@ def test_wan_480p(usv):
     _attention_parity(usv, q, k, v, wl.N, wl.k_per_head(), 64, 1)
 
 
+@pytest.mark.parametrize("name", ["seq_99k", "seq_131k", "seq_193k"])
+def test_sequence_length_sweep(usv, name):
+    """The paper's speedup-vs-length points (about 99k / 131k / 193k tokens) at keep 5 %: selection
+    in full (rows of 1560 / 2048 / 3023 scores: both selection kernels), attention on samples."""
+    wl = ui.workload(name)
+    q, k, v = ui.make_qkv(wl, device=DEV, layout="bhnd")
+    _attention_parity(usv, q, k, v, wl.N, wl.k_per_head(), 24, 50 + wl.index)
+
+
 def test_wan_14b_720p(usv):
     wl = ui.workload("wan14b_720p")
     q, k, v = ui.make_qkv(wl, device=DEV)

@@ -184,6 +184,15 @@ WORKLOADS = [
     Workload("hunyuan_720p", 4, 2, 24, 128, (33, 45, 80), (100, 25, 10, 5),
              merge_part=(1, 1, 2), merge_percent=25,
              note="HunyuanVideo 720p-shaped CFG pair, per-head keep sweep, 25% merge"),
+    # Sequence-length sweep at the Wan2.1-1.3B head shape: the token counts of the paper's
+    # speedup-vs-length study (about 99k / 131k / 193k tokens = 61 / 81 / 121 frames of a 60 x 104
+    # latent grid before patchify), at its attention sparsity of 0.95 (keep 5 % of the key blocks).
+    Workload("seq_99k", 5, 1, 12, 128, (16, 60, 104), (5,),
+             note="length sweep, 99 840 tokens, 1560 blocks, keep 5%"),
+    Workload("seq_131k", 6, 1, 12, 128, (21, 60, 104), (5,),
+             note="length sweep, 131 040 tokens, 2048 blocks, keep 5%"),
+    Workload("seq_193k", 7, 1, 12, 128, (31, 60, 104), (5,),
+             note="length sweep, 193 440 tokens, 3023 blocks, keep 5%"),
 ]
 
 
