@@ -65,7 +65,9 @@ const char* usv_build_info(void);
  *     scores[b,h,I,J] = < mean_q[b,h,I,:], mean_k[b,h,J,:] > / sqrt(d)          (fp32).
  *
  * q: bf16 view [B,H,Nq,d], k: bf16 view [B,H,Nk,d]; d in {64,128}.
- * scores: fp32 [B,H,NBq,NBk] contiguous (written).  ws: pooled means, see *_workspace().
+ * scores: fp32 [B,H,NBq,NBk] contiguous (written).  ws: pooled means (and, at d = 128, the bf16
+ * operand planes of the tensor-core product, which is accumulated in fp32 from a three-way split
+ * of every fp32 mean and is fp32-accurate), see *_workspace().
  */
 size_t usv_block_scores_workspace(int B, int H, int Nq, int Nk, int d);
 int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void* q, const usv_strides* sq,
@@ -86,7 +88,8 @@ int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void* q, const u
  *   - Same arguments and results as usv_block_scores minus ws/ws_bytes.  Nothing is allocated
  *     or freed, by the CUDA runtime or any other library.
  *   - The request is rejected (USV_ERR_WORKSPACE, nothing launched) when
- *     usv_block_scores_workspace(B,H,Nq,Nk,d) exceeds USV_NOALLOC_SCRATCH_BYTES.
+ *     the pooled means of q and k (B*H*(NBq + NBk)*d fp32 values, each tensor rounded up to
+ *     256 bytes) exceed USV_NOALLOC_SCRATCH_BYTES.
  *   - The first call on each device looks up the array's device address (a one-off, synchronous
  *     runtime query with that device current).  Make that first call before starting any
  *     stream capture on the device.

@@ -5,7 +5,7 @@
 //   scores_kernel : fp32 CUDA-core NT GEMM per (b,h), 64x64 output tile, 4x4 per thread.
 //                   Kept in fp32 (not bf16 tensor cores) because the result decides an integer
 //                   (the top-k set) that is compared with an fp64 evaluation.
-#include "usv_common.cuh"
+#include "usv_scores.cuh"
 
 namespace usv {
 
@@ -128,8 +128,10 @@ __global__ void __launch_bounds__(256) scores_kernel(const float* __restrict__ q
 extern "C" size_t usv_block_scores_workspace(int B, int H, int Nq, int Nk, int d) {
     if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || d <= 0) return 0;
     const size_t nbq = usv::ceil_div(Nq, USV_BLOCK), nbk = usv::ceil_div(Nk, USV_BLOCK);
+    // pooled means of q and k; at d = 128 also the bf16 planes of the tensor-core scores kernel
     return usv::align_up((size_t)B * H * nbq * d * sizeof(float), 256) +
-           usv::align_up((size_t)B * H * nbk * d * sizeof(float), 256);
+           usv::align_up((size_t)B * H * nbk * d * sizeof(float), 256) +
+           (d == 128 ? usv::scores_tc_bytes(B * H, (int)nbq, (int)nbk) : 0);
 }
 
 extern "C" int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void* q,
@@ -168,6 +170,10 @@ extern "C" int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void*
     else pool_kernel<64><<<pg, 128, 0, st>>>(a);
     USV_CHECK_LAUNCH("pool_kernel");
 
+    if (d == 128) {
+        void* mem = reinterpret_cast<char*>(kbar) + align_up((size_t)B * H * NBk * d * sizeof(float), 256);
+        return launch_scores_tc(qbar, kbar, scores, B * H, NBq, NBk, 1.0f / sqrtf((float)d), mem, st);
+    }
     dim3 sg(ceil_div(NBk, 64), ceil_div(NBq, 64), B * H);
     scores_kernel<<<sg, 256, 0, st>>>(qbar, kbar, scores, NBq, NBk, d, 1.0f / sqrtf((float)d));
     USV_CHECK_LAUNCH("scores_kernel");
@@ -219,7 +225,8 @@ extern "C" int usv_block_scores_noalloc(int B, int H, int Nq, int Nk, int d, con
     if ((rc = check_view("k", k, sk, d)) != USV_OK) return rc;
     if (scores == nullptr) return fail(USV_ERR_INVALID_ARG, "block_scores_noalloc: null scores");
     if (!aligned16(scores)) return fail(USV_ERR_UNSUPPORTED, "block_scores_noalloc: scores not 16-byte aligned");
-    const size_t need = usv_block_scores_workspace(B, H, Nq, Nk, d);
+    const size_t need = align_up((size_t)B * H * ceil_div(Nq, USV_BLOCK) * d * sizeof(float), 256) +
+                        align_up((size_t)B * H * ceil_div(Nk, USV_BLOCK) * d * sizeof(float), 256);
     if (need > (size_t)USV_NOALLOC_SCRATCH_BYTES)
         return fail(USV_ERR_WORKSPACE,
                     "block_scores_noalloc: needs %zu bytes of scratch, the built-in array holds %u; "
