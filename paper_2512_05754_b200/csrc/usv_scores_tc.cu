@@ -95,7 +95,12 @@ scores_tc_kernel(const Args m, const __grid_constant__ Maps maps) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.y;
     const int i0 = blockIdx.x * 128;
-    const int T = m.NBk_pad / 128;   // key-block tiles
+    // key-block tiles [t_lo, t_hi) of this CTA: the column range is split over blockIdx.z so that
+    // short problems still fill the GPU
+    const int t_all = m.NBk_pad / 128;
+    const int t_per = (t_all + gridDim.z - 1) / gridDim.z;
+    const int t_lo = min(t_all, (int)blockIdx.z * t_per);
+    const int T = min(t_all, t_lo + t_per) - t_lo;
 
     if (threadIdx.x == 0) {
         mbar_init(bar(B_AFULL), 4);
@@ -132,8 +137,8 @@ scores_tc_kernel(const Args m, const __grid_constant__ Maps maps) {
                 mbar_expect_tx(bar(B_BFULL + s), STAGE_BYTES);
 #pragma unroll
                 for (int p = 0; p < NPL; ++p) {
-                    tma_load_2d(dst + p * PLANE_BYTES, &maps.b[p], bar(B_BFULL + s), 0, row0 + t * 128);
-                    tma_load_2d(dst + p * PLANE_BYTES + 16384, &maps.b[p], bar(B_BFULL + s), 64, row0 + t * 128);
+                    tma_load_2d(dst + p * PLANE_BYTES, &maps.b[p], bar(B_BFULL + s), 0, row0 + (t_lo + t) * 128);
+                    tma_load_2d(dst + p * PLANE_BYTES + 16384, &maps.b[p], bar(B_BFULL + s), 64, row0 + (t_lo + t) * 128);
                 }
             }
             __syncwarp();
@@ -218,7 +223,7 @@ scores_tc_kernel(const Args m, const __grid_constant__ Maps maps) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) tbuf[lane * 33 + j] = __uint_as_float(sr[j]) * m.scale;
                 __syncwarp();
-                const int col = t * 128 + ch * 32 + lane;
+                const int col = (t_lo + t) * 128 + ch * 32 + lane;
                 if (col < m.NBk)
                     for (int rr = 0; rr < nrows; ++rr) out[(int64_t)rr * m.NBk + col] = tbuf[rr * 33 + lane];
                 __syncwarp();
@@ -283,7 +288,10 @@ int launch_scores_tc(const float* qbar, const float* kbar, float* scores, int BH
     }
     e = cudaFuncSetAttribute(sc::scores_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sc::SMEM_BYTES);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "block_scores: smem attribute: %s", cudaGetErrorString(e));
-    dim3 grid(m.NBq_pad / 128, BH);
+    const int ctas = (m.NBq_pad / 128) * BH, t_all = m.NBk_pad / 128;
+    int nz = (296 + ctas - 1) / ctas;          // aim at two CTAs' worth of work per SM
+    nz = nz < 1 ? 1 : (nz > t_all ? t_all : nz);
+    dim3 grid(m.NBq_pad / 128, BH, nz);
     sc::scores_tc_kernel<<<grid, 192, sc::SMEM_BYTES, st>>>(m, maps);
     USV_CHECK_LAUNCH("scores_tc_kernel");
     return USV_OK;
