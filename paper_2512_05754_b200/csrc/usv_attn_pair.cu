@@ -134,35 +134,23 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const bool live = Iq >= 0 && row < N;
 
     // ---- set-up: barriers, TMEM, the pair's key-block list -> shared memory, Q -> TMEM
-    if (threadIdx.x == 0) {
-        mbar_init(bar(B_QFULL), NSOFT / 32);       // one arrival per softmax warp
-        for (int s = 0; s < KSTAGES; ++s) {
-            mbar_init(bar(B_KFULL + s), 1);
-            mbar_init(bar(B_KEMPTY + s), 1);
+    if (warp == 0) {
+        // one barrier per lane (a single thread initialising all of them takes ~1000 cycles)
+        uint32_t count = 1;                                           // K/V stages, SFULL, PFREE, OFULL
+        if (lane == B_QFULL || lane == B_EPI || lane == B_EPI + 1) count = NSOFT / 32;   // one arrival per softmax warp
+        // SFREE / PFULL: one arrival per warp of the two groups of a tile.  PV(t) commits to
+        // PFREE[t & 1]: each waiter then sees every phase of the barrier it waits on (a thread that
+        // skipped a phase could not tell it from the one two before).
+        if (lane == B_SFREE || lane == B_SFREE + 1 || lane == B_PFULL || lane == B_PFULL + 1) count = 8;
+        // REF / EPI: rendezvous of the softmax threads after the first bounded wait: mbarriers, so
+        // that they too can give up (a bar.sync would hang if one thread had left its loop)
+        if (lane == B_REF || lane == B_REF + 1) count = 2;            // the two warps of the owning group on a side
+        if (lane < B_COUNT) mbar_init(bar(lane), count);
+        if (lane == 0) {
+            *s_abort = 0;
+            s_flag[0] = 0;
+            s_flag[1] = 0;
         }
-        for (int s = 0; s < VSTAGES; ++s) {
-            mbar_init(bar(B_VFULL + s), 1);
-            mbar_init(bar(B_VEMPTY + s), 1);
-        }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(B_SFULL + s), 1);
-            mbar_init(bar(B_SFREE + s), 8);         // one arrival per warp of the two groups
-            mbar_init(bar(B_PFULL + s), 8);
-        }
-        // PV(t) commits to PFREE[t & 1]: each waiter then sees every phase of the barrier it waits on
-        // (a thread that skipped a phase could not tell it from the one two before)
-        mbar_init(bar(B_PFREE), 1);
-        mbar_init(bar(B_PFREE + 1), 1);
-        mbar_init(bar(B_OFULL), 1);
-        // rendezvous of the softmax threads after the first bounded wait: mbarriers, so that they
-        // too can give up (a bar.sync would hang if one thread had left its loop)
-        mbar_init(bar(B_REF), 2);                   // the two warps of the owning group on a side
-        mbar_init(bar(B_REF + 1), 2);
-        mbar_init(bar(B_EPI), NSOFT / 32);
-        mbar_init(bar(B_EPI + 1), NSOFT / 32);
-        *s_abort = 0;
-        s_flag[0] = 0;
-        s_flag[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == W_MMA) {
