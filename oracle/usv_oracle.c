@@ -31,6 +31,10 @@
  *   usvo_merge_positions    Sec. 3.3, Eq. 14: merged order [U ascending || B ascending].
  *   usvo_merge_apply        Sec. 3.3, Eq. 12-13: mean aggregation into destinations.
  *   usvo_unmerge            Sec. 3.3, Eq. 15: copy back by stored plan.
+ *   usvo_key_marginal       Sec. 3.4, Eq. 16: attention weights (here: of the block-masked
+ *                           attention of Eq. 5) averaged over heads and queries.
+ *   usvo_entropy            Sec. 3.4, Eq. 17: entropy of that marginal, normalised by log N.
+ *   usvo_allocate           Sec. 3.4, Eq. 18-19: w = (1-h)^gamma, rho_l = clip(rho_bar w_l / mean w).
  */
 #include <math.h>
 #include <stdint.h>
@@ -474,5 +478,69 @@ void usvo_unmerge(const uint16_t* y, int B, int N, int C, int Nm, const int32_t*
     for (int64_t bn = 0; bn < (int64_t)B * N; ++bn) {
         int b = (int)(bn / N);
         memcpy(out + bn * C, y + ((int64_t)b * Nm + pos[bn]) * C, sizeof(uint16_t) * (size_t)C);
+    }
+}
+
+/* ---------------------------------------------------------------- entropy-aware scheduler */
+
+/* Eq. 16: abar[b][j] = 1/(H N) sum_h sum_i A(h,i,j), A = row-wise softmax of the scaled logits
+ * over the valid keys of the selected key blocks (Eq. 5), zero elsewhere.  marg: [B,N]. */
+void usvo_key_marginal(const uint16_t* q, const int64_t* sq, const uint16_t* k, const int64_t* sk,
+                       int B, int H, int N, int d, const int32_t* sel, const int32_t* k_per_head,
+                       int kmax, double scale, double* marg) {
+    int NB = (N + USVO_BS - 1) / USVO_BS;
+    for (int64_t x = 0; x < (int64_t)B * N; ++x) marg[x] = 0.0;
+    double* a = (double*)malloc(sizeof(double) * (size_t)N);
+    int32_t* idx = (int32_t*)malloc(sizeof(int32_t) * (size_t)N);
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h)
+            for (int i = 0; i < N; ++i) {
+                const int32_t* row = sel + (((int64_t)b * H + h) * NB + i / USVO_BS) * kmax;
+                int nk = 0;
+                double mx = -INFINITY;
+                for (int t = 0; t < k_per_head[h]; ++t) {
+                    int J = row[t];
+                    if (J < 0) continue;
+                    for (int j = J * USVO_BS; j < (J + 1) * USVO_BS && j < N; ++j) {
+                        double acc = 0.0;
+                        for (int e = 0; e < d; ++e)
+                            acc += bf16_val(q[b * sq[0] + h * sq[1] + i * sq[2] + e]) *
+                                   bf16_val(k[b * sk[0] + h * sk[1] + j * sk[2] + e]);
+                        a[nk] = acc * scale;
+                        idx[nk] = j;
+                        mx = a[nk] > mx ? a[nk] : mx;
+                        ++nk;
+                    }
+                }
+                double sum = 0.0;
+                for (int c = 0; c < nk; ++c) {
+                    a[c] = exp(a[c] - mx);
+                    sum += a[c];
+                }
+                for (int c = 0; c < nk; ++c) marg[(int64_t)b * N + idx[c]] += a[c] / sum;
+            }
+    for (int64_t x = 0; x < (int64_t)B * N; ++x) marg[x] /= (double)H * (double)N;
+    free(a);
+    free(idx);
+}
+
+/* Eq. 17: h = -(1/log N) sum_j abar(j) log abar(j), with 0 log 0 = 0. */
+double usvo_entropy(const double* marg, int N) {
+    double s = 0.0;
+    for (int j = 0; j < N; ++j)
+        if (marg[j] > 0.0) s -= marg[j] * log(marg[j]);
+    return N > 1 ? s / log((double)N) : 0.0;
+}
+
+/* Eq. 18-19 for the L layers of one step. */
+void usvo_allocate(const double* h, int L, double gamma, double rho_bar, double rho_min,
+                   double rho_max, double* rho) {
+    double mean = 0.0;
+    for (int l = 0; l < L; ++l) mean += pow(1.0 - h[l], gamma);
+    mean /= (double)L;
+    for (int l = 0; l < L; ++l) {
+        double w = pow(1.0 - h[l], gamma);
+        double r = rho_bar * w / mean;
+        rho[l] = r < rho_min ? rho_min : (r > rho_max ? rho_max : r);
     }
 }

@@ -25,7 +25,7 @@ __all__ = [
     "BS", "build", "num_threads", "bf16_bits", "bf16_to_f64", "round_to_bf16", "block_pool",
     "block_scores", "select_blocks", "dense_masked_attn", "sparse_attn", "destination_mask",
     "merge_descriptors", "merge_match", "merge_select", "merge_positions", "merge_plan",
-    "merge_apply", "unmerge", "all_query_blocks", "keep_count",
+    "merge_apply", "unmerge", "all_query_blocks", "keep_count", "key_marginal", "entropy", "allocate",
 ]
 
 
@@ -49,6 +49,7 @@ def _L():
         _lib = ctypes.CDLL(_LIB)
         _lib.usvo_merge_positions.restype = ctypes.c_int
         _lib.usvo_num_threads.restype = ctypes.c_int
+        _lib.usvo_entropy.restype = ctypes.c_double
     return _lib
 
 
@@ -299,4 +300,37 @@ def unmerge(y, pos):
     N = p.shape[1]
     out = np.empty((B, N, C), dtype=np.uint16)
     _L().usvo_unmerge(_p(a), B, N, C, Nm, _p(p), _p(out))
+    return out
+
+
+# ------------------------------------------------------------------ entropy-aware scheduler
+
+
+def key_marginal(q, k, N, sel, k_per_head, scale=None):
+    """Eq. 16 for the block-masked attention: fp64 [B,N], each row sums to one."""
+    qa, sq = _strided(q)
+    ka, sk = _strided(k)
+    B, H, _, d = qa.shape
+    sel = np.ascontiguousarray(sel, dtype=np.int32)
+    kph = np.ascontiguousarray(k_per_head, dtype=np.int32)
+    scale = 1.0 / np.sqrt(d) if scale is None else float(scale)
+    out = np.empty((B, int(N)), dtype=np.float64)
+    s3 = lambda s: (ctypes.c_int64 * 3)(*s)
+    _L().usvo_key_marginal(_p(qa), s3(sq), _p(ka), s3(sk), B, H, int(N), d, _p(sel), _p(kph), sel.shape[3],
+                           ctypes.c_double(scale), _p(out))
+    return out
+
+
+def entropy(marg):
+    """Eq. 17 per batch element: fp64 [B]."""
+    m = np.ascontiguousarray(marg, dtype=np.float64)
+    return np.array([_L().usvo_entropy(_p(m[b]), m.shape[1]) for b in range(m.shape[0])])
+
+
+def allocate(h, gamma, rho_bar, rho_min, rho_max):
+    """Eq. 18-19: per-layer ratios from per-layer entropies."""
+    h = np.ascontiguousarray(h, dtype=np.float64)
+    out = np.empty_like(h)
+    _L().usvo_allocate(_p(h), h.shape[0], ctypes.c_double(gamma), ctypes.c_double(rho_bar),
+                       ctypes.c_double(rho_min), ctypes.c_double(rho_max), _p(out))
     return out
