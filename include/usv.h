@@ -187,6 +187,32 @@ int usv_token_merge(int B, int N, int C, const void* x, int Hm, int dm, const vo
 int usv_token_unmerge(int B, int N, int Nm, int C, const void* y_merged, const int32_t* pos,
                       void* y, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Entropy-aware scheduler inputs (Sec. 3.4).
+ *
+ * usv_attn_entropy: key marginal of the block-masked attention weights averaged over heads and
+ * queries (Eq. 16), abar[b,j] = 1/(H N) sum_h sum_i A(h,i,j), and its entropy normalised by log N
+ * (Eq. 17), h[b] in [0,1].  A is recomputed as exp(scale <q_i,k_j> - lse_i) from the
+ * log-sum-exp that usv_sparse_attn_fwd wrote for the same q, k, sel.
+ *
+ * q,k: bf16 views [B,H,N,d], d in {64,128}.  sel / k_per_head (HOST) / kmax / scale: as passed to
+ * usv_sparse_attn_fwd.  lse: fp32 [B,H,N] from that call.  key_marginal: fp32 [B,N] (written;
+ * sums to 1 per batch element up to rounding).  entropy: fp32 [B] (written).  The sums use fp32
+ * atomic adds: results are reproducible to rounding, not bit for bit.
+ */
+int usv_attn_entropy(int B, int H, int N, int d, const void* q, const usv_strides* sq,
+                     const void* k, const usv_strides* sk, const int32_t* sel,
+                     const int32_t* k_per_head, int kmax, const float* lse, float scale,
+                     float* key_marginal, float* entropy, void* stream);
+
+/* Entropy-aware allocation over the L layers of one step (Eq. 18-19), plain host arithmetic:
+ *     w_l = (1 - h_l)^gamma ,   rho_l = clip(rho_min, rho_max, rho_bar * w_l / mean_l'(w_l')).
+ * entropy, rho: HOST arrays of L floats; gamma >= 1; every h_l in [0,1].  If every w_l is zero
+ * each layer keeps rho_bar (clipped).  Serves the attention and the token ratio alike.
+ */
+int usv_allocate_sparsity(int L, const float* entropy, float gamma, float rho_bar, float rho_min,
+                          float rho_max, float* rho);
+
 #ifdef __cplusplus
 }
 #endif

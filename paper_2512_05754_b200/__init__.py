@@ -6,5 +6,6 @@ device memory and streams.
 """
 from .binding import (  # noqa: F401
     USVError, lib, lib_path, block_scores, block_scores_noalloc, select_blocks, sparse_attn_fwd, token_merge,
-    token_unmerge, MergePlan, workspace_status, sparse_attn_fallbacks, build_info, BLOCK,
+    token_unmerge, MergePlan, workspace_status, sparse_attn_fallbacks, build_info, BLOCK, attn_entropy,
+    allocate_sparsity,
 )

@@ -258,3 +258,35 @@ def token_unmerge(y_merged, pos, out=None):
     _check(lib().usv_token_unmerge(B, N, Nm, C, _ptr(y_merged), _ptr(pos), _ptr(out),
                                    _stream(y_merged.device)), "usv_token_unmerge")
     return out
+
+
+def attn_entropy(q, k, sel, k_per_head, lse, N=None, scale=0.0):
+    """Key marginal [B,N] of the block-masked attention weights averaged over heads and queries,
+    and its entropy normalised by log N [B].  `lse` is the log-sum-exp of sparse_attn_fwd for the
+    same q, k, sel."""
+    sq, sk = _view(q, "q"), _view(k, "k")
+    B, H, n, d = q.shape
+    N = n if N is None else int(N)
+    if sel.dtype != torch.int32 or not sel.is_contiguous() or not sel.is_cuda:
+        raise ValueError("sel must be a contiguous CUDA int32 tensor")
+    if lse.dtype != torch.float32 or not lse.is_contiguous() or tuple(lse.shape) != (B, H, N):
+        raise ValueError("lse must be a contiguous CUDA fp32 [B,H,N] tensor")
+    karr, _ = _k_array(k_per_head, H)
+    marg = torch.empty((B, N), dtype=torch.float32, device=q.device)
+    ent = torch.empty((B,), dtype=torch.float32, device=q.device)
+    _check(lib().usv_attn_entropy(B, H, N, d, _ptr(q), ctypes.byref(sq), _ptr(k), ctypes.byref(sk), _ptr(sel),
+                                  karr, sel.shape[3], _ptr(lse), ctypes.c_float(scale), _ptr(marg), _ptr(ent),
+                                  _stream(q.device)), "usv_attn_entropy")
+    return marg, ent
+
+
+def allocate_sparsity(entropy, gamma, rho_bar, rho_min, rho_max):
+    """Per-layer ratios from per-layer entropies (host arithmetic): list of floats."""
+    h = [float(x) for x in entropy]
+    L = len(h)
+    inp = (ctypes.c_float * L)(*h)
+    out = (ctypes.c_float * L)()
+    _check(lib().usv_allocate_sparsity(L, inp, ctypes.c_float(gamma), ctypes.c_float(rho_bar),
+                                       ctypes.c_float(rho_min), ctypes.c_float(rho_max), out),
+           "usv_allocate_sparsity")
+    return list(out)
