@@ -41,6 +41,9 @@ CASES = [
     ("tiny", 1, 2, (4, 16, 16), 64, "bhnd", [4, 4]),
     ("ragged_d128", 2, 3, (10, 10, 10), 128, "bnhd", [3, 16, 7]),
     ("ragged_d64", 1, 4, (5, 23, 39), 64, "bhnd", [1, 71, 10, 35]),
+    # degenerate sizes of the paired kernel: one partial block (a pair without partner); three blocks
+    ("single_block", 1, 2, (1, 5, 10), 128, "bhnd", [1, 1]),
+    ("three_blocks", 1, 1, (1, 12, 15), 128, "bnhd", [2]),
 ]
 
 
