@@ -117,6 +117,32 @@ def test_keep_all_matches_dense_attention(usv):
     assert mx <= MAX_ABS and rl2 <= 3e-3
 
 
+@pytest.mark.parametrize("kb,expect_fallback", [(20.0, False), (64.0, True)])
+def test_fixed_reference_range_and_exact_recomputation(usv, kb, expect_fallback):
+    """The tcgen05 kernel fixes a row's softmax reference at its first key block.  Logits of a later
+    block ~82 octaves above it stay inside the fp32/bf16 exponent range (no recomputation);
+    ~260 octaves above it overflow, the query blocks are reported and recomputed exactly.  Either
+    way the result must match the oracle."""
+    B, H, N, d = 1, 1, 256, 128
+    g = torch.Generator().manual_seed(3)
+    q = torch.zeros(B, H, N, d); q[..., 0] = 32.0
+    k = torch.zeros(B, H, N, d); k[:, :, 192:, 0] = kb          # block 3: logit 32*kb/sqrt(128)
+    v = torch.randn(B, H, N, d, generator=g)
+    q, k, v = (t.to(torch.bfloat16) for t in (q, k, v))
+    sel = torch.arange(4, dtype=torch.int32).expand(B, H, 4, 4).contiguous()
+    o, o32, lse = usv.sparse_attn_fwd(q.to(_dev()), k.to(_dev()), v.to(_dev()), sel.to(_dev()), [4], N=N,
+                                      return_f32=True, return_lse=True)
+    torch.cuda.synchronize()
+    assert usv.workspace_status() == 0
+    nfb = usv.sparse_attn_fallbacks()
+    assert nfb == (4 if expect_fallback else 0)
+    o_ref, lse_ref = oracle.sparse_attn(q, k, v, N, sel.numpy(), [4])
+    mx, rl2 = attn_errors(o32.cpu().numpy(), o_ref.reshape(B, H, N, d))
+    assert mx <= MAX_ABS and rl2 <= 3e-3          # white-noise values: see test_keep_all_matches_dense_attention
+    assert np.abs(lse.cpu().numpy() - lse_ref.reshape(B, H, N)).max() <= 2e-3 * max(1.0, np.abs(lse_ref).max())
+    assert torch.isfinite(o.float()).all()
+
+
 def test_select_kernel_exact_on_tied_scores(usv):
     """Integer-valued scores with many exact ties: the tie rule must hold bit-exactly."""
     g = torch.Generator().manual_seed(11)
