@@ -5,8 +5,8 @@
 // therefore owns TWO query blocks (rows 0-63 = block A, rows 64-127 = block B of one head) and
 // walks the ascending UNION of their two key-block lists, two key blocks (128 keys) per tile:
 //
-//     S[128 q x 128 keys]  = Q . K_tile^T      tcgen05.mma, A = Q resident in TMEM, B = K in smem
-//     O[128 q x 128 d]    += P . V_tile        tcgen05.mma, A = P (bf16) in TMEM,   B = V in smem
+//     S[128 q x 128 keys]  = Q . K_tile^T      tcgen05.mma, A = Q in smem,        B = K in smem
+//     O[128 q x 128 d]    += P . V_tile        tcgen05.mma, A = P (bf16) in TMEM, B = V in smem
 //
 // A key block that only one of the two lists holds is masked for the other half of the rows
 // (its softmax weights are written as zero), so the result is exactly the per-block selection.
@@ -23,16 +23,19 @@
 //
 // CTA = 19 warps.  Warps 0-15 are four softmax/epilogue warpgroups that share the 128 rows
 // (thread r of every group <-> TMEM lane r <-> query row r).  Group g works on the tiles of
-// parity g >> 1 (S/P buffer g >> 1) and there on key block g & 1 of the tile (64 logit columns),
-// so two tiles are in the softmax stage at a time, each spread over 256 threads.  Warp 16 is the
-// K producer (TMA), warp 17 the MMA issuer and TMEM owner, warp 18 the V producer.
+// parity g >> 1 and there on key block g & 1 of the tile (64 logit columns), so two tiles are in
+// the softmax stage at a time, each spread over 256 threads.  Warp 16 is the K producer (TMA; it
+// also fetches the pair's Q rows), warp 17 the MMA issuer and TMEM owner, warp 18 the V producer.
 //
-// TMEM holds Q, two S buffers, O and ONE P buffer.  A softmax thread gives its S buffer back as
-// soon as the logits are in its registers (S of the tile after next is then computed while it
-// exponentiates), and writes P once the P.V product of the tile before has finished reading the
-// P buffer.  There is one commit after S(t) (publishes S, frees the K stage) and one after
-// PV(t) (frees the P buffer and the V stage).  All waits are bounded; a wait that
-// gives up sets the device status word and every role leaves its loop.
+// TMEM holds O and THREE S buffers; tile t uses buffer t mod 3.  The weights P(t) are written
+// back, as bf16 pairs, into the columns their logits came from, so a buffer goes
+// S(t) -> P(t) -> S(t + 3) without a hand-back: P.V(t) is issued before S(t + 3), and the tensor
+// pipe runs its MMAs in issue order.  With three buffers a finished S tile is always waiting
+// when a softmax group comes free, and a finished P tile when the pipe does.  Every barrier has
+// one set of waiters that sees each of its phases (SFULL/PFULL are indexed by t mod 6: the two
+// tile parities of a buffer wait on different barriers; a waiter that skipped a phase could not
+// tell it from the one two before).  All waits are bounded; a wait that gives up sets the device
+// status word and every role leaves its loop.
 #include "usv_attn.cuh"
 #include "usv_tcgen05.cuh"
 
@@ -49,13 +52,15 @@ constexpr int KSTAGES = 2;                      // K tile stages
 constexpr int VSTAGES = 3;                      // V tile stages
 constexpr int MAX_NB = 4096;                    // key blocks per sequence this kernel covers
 constexpr uint32_t TILE_BYTES = KT * D * 2;     // 32 KB: [d-half][128 keys][128 B]
-constexpr uint32_t SM_K = 0;
+constexpr int SBUF = 3;                         // S/P buffers in TMEM
+constexpr uint32_t SM_Q = 0;                    // the pair's 128 query rows, same layout as a K tile
+constexpr uint32_t SM_K = SM_Q + TILE_BYTES;
 constexpr uint32_t SM_V = SM_K + KSTAGES * TILE_BYTES;
 constexpr uint32_t SM_BAR = SM_V + VSTAGES * TILE_BYTES;
 // barrier slots (8 bytes each)
 enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = B_KFULL + KSTAGES, B_VFULL = B_KEMPTY + KSTAGES,
-       B_VEMPTY = B_VFULL + VSTAGES, B_SFULL = B_VEMPTY + VSTAGES, B_SFREE = B_SFULL + 2,
-       B_PFULL = B_SFREE + 2, B_PFREE = B_PFULL + 2, B_OFULL = B_PFREE + 2, B_REF, B_EPI = B_REF + 2, B_COUNT = B_EPI + 2 };
+       B_VEMPTY = B_VFULL + VSTAGES, B_SFULL = B_VEMPTY + VSTAGES, B_PFULL = B_SFULL + 2 * SBUF,
+       B_OFULL = B_PFULL + 2 * SBUF, B_REF, B_EPI = B_REF + 2, B_COUNT = B_EPI + 2 };
 static_assert(B_COUNT <= 32, "barrier area");
 constexpr uint32_t SM_MISC = SM_BAR + 8 * 32;            // tmem base, abort flag, flags, union size
 constexpr uint32_t SM_LIST = SM_MISC + 64;               // int[MAX_NB]: (key block << 2) | in-A | in-B << 1
@@ -64,10 +69,10 @@ constexpr uint32_t SM_SUM = SM_REFV + 128 * 4;           // float[NWG][128]: par
 constexpr uint32_t SM_TOTAL = SM_SUM + NWG * 128 * 4;
 constexpr size_t SMEM_BYTES = SM_TOTAL + 1024;           // + slack for 1024-byte alignment
 
-// TMEM columns: Q (bf16 pairs) | S buffer 0 | S buffer 1 | O | P (bf16 pairs)
+// TMEM columns: O | S/P buffer 0 | S/P buffer 1 | S/P buffer 2
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t TQ = 0, TS = 64, TO = TS + 2 * 128, TP = TO + 128;
-static_assert(TP + 64 <= TMEM_COLS, "TMEM budget");
+constexpr uint32_t TO = 0, TS = 128;
+static_assert(TS + SBUF * 128 <= TMEM_COLS, "TMEM budget");
 
 constexpr int NSOFT = NWG * 128;   // softmax threads
 constexpr int NTHREADS = NSOFT + 96;
@@ -75,7 +80,7 @@ constexpr int W_TMA = NSOFT / 32, W_MMA = NSOFT / 32 + 1, W_TMA_V = NSOFT / 32 +
 __device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory"); }
 
 struct Maps {
-    CUtensorMap k, v;
+    CUtensorMap q, k, v;
 };
 
 // exp2 of 32 scaled logits -> 16 packed bf16 pairs; adds the (unrounded) weights to the two
@@ -133,15 +138,13 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     const int row = Iq * USV_BLOCK + (r & 63);
     const bool live = Iq >= 0 && row < N;
 
-    // ---- set-up: barriers, TMEM, the pair's key-block list -> shared memory, Q -> TMEM
+    // ---- set-up: barriers, TMEM, the pair's key-block list -> shared memory
     if (warp == 0) {
         // one barrier per lane (a single thread initialising all of them takes ~1000 cycles)
-        uint32_t count = 1;                                           // K/V stages, SFULL, PFREE, OFULL
-        if (lane == B_QFULL || lane == B_EPI || lane == B_EPI + 1) count = NSOFT / 32;   // one arrival per softmax warp
-        // SFREE / PFULL: one arrival per warp of the two groups of a tile.  PV(t) commits to
-        // PFREE[t & 1]: each waiter then sees every phase of the barrier it waits on (a thread that
-        // skipped a phase could not tell it from the one two before).
-        if (lane == B_SFREE || lane == B_SFREE + 1 || lane == B_PFULL || lane == B_PFULL + 1) count = 8;
+        uint32_t count = 1;                                           // Q, K/V stages, SFULL, OFULL
+        if (lane == B_EPI || lane == B_EPI + 1) count = NSOFT / 32;   // one arrival per softmax warp
+        // PFULL: one arrival per warp of the two groups of a tile
+        if (lane >= B_PFULL && lane < B_PFULL + 2 * SBUF) count = 8;
         // REF / EPI: rendezvous of the softmax threads after the first bounded wait: mbarriers, so
         // that they too can give up (a bar.sync would hang if one thread had left its loop)
         if (lane == B_REF || lane == B_REF + 1) count = 2;            // the two warps of the owning group on a side
@@ -159,12 +162,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     const int* plist = a.lists + b * a.list_batch + a.list_off[h] + (int64_t)pair * list_stride(kh, NB);
-    uint4 qv[4];   // this thread's quarter of its query row (32 of the 128 bf16)
     if (warp < W_TMA) {
-        const uint4* src = reinterpret_cast<const uint4*>(a.q + b * a.sq.sb + h * a.sq.sh +
-                                                          (int64_t)row * a.sq.sn + grp * 32);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) qv[i] = live ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
         // the pair's union key-block list (built by the plan kernels) -> shared memory
         const int lstride = (int)list_stride(kh, NB);
         for (int i = threadIdx.x; i < lstride; i += NSOFT) {
@@ -177,19 +175,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     fence_after();
     const uint32_t tmem = *s_tmem;
     const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    if (warp < W_TMA) {
-        // this thread's part of its query row -> TMEM (two bf16 of consecutive d per column)
-        uint32_t q[16];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            q[4 * i] = qv[i].x; q[4 * i + 1] = qv[i].y; q[4 * i + 2] = qv[i].z; q[4 * i + 3] = qv[i].w;
-        }
-        tmem_st16(lane_base + TQ + grp * 16, q);
-        tmem_wait_st();
-        fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(B_QFULL));
-    }
     const int nU = *s_nu;
     const int T = (nU + 1) >> 1;   // 128-key tiles
 
@@ -197,6 +182,16 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
         // ===== K producer (whole warp in the loop, one elected lane issues) =====================
         // K and V have a producer warp each: a K stage comes back as soon as S is computed, long
         // before the V stage of the same tile does, and must not queue behind it.
+        if (T > 0 && elect_one()) {
+            // the pair's query rows; a block without a partner reads rows past the end (zero fill)
+            const int ra = IA * USV_BLOCK, rb = (IB >= 0 ? IB : NB) * USV_BLOCK;
+            mbar_expect_tx(bar(B_QFULL), TILE_BYTES);
+            tma_load_4d(base + SM_Q, &maps.q, bar(B_QFULL), 0, ra, h, b);
+            tma_load_4d(base + SM_Q + 8192, &maps.q, bar(B_QFULL), 0, rb, h, b);
+            tma_load_4d(base + SM_Q + 16384, &maps.q, bar(B_QFULL), 64, ra, h, b);
+            tma_load_4d(base + SM_Q + 24576, &maps.q, bar(B_QFULL), 64, rb, h, b);
+        }
+        __syncwarp();
         for (int t = 0; t < T; ++t) {
             const int s = t % KSTAGES;
             const uint32_t ph = (t / KSTAGES) & 1;
@@ -234,63 +229,57 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     } else if (warp == W_MMA) {
         // ===== MMA issuer (whole warp in the loop, one elected lane issues); TMEM owner =========
         if (T > 0) {
-            constexpr uint32_t IDESC_S = instr_desc(128, KT, 0, 0);    // Q (TMEM) x K (K-major)
+            constexpr uint32_t IDESC_S = instr_desc(128, KT, 0, 0);    // Q (K-major) x K (K-major)
             constexpr uint32_t IDESC_O = instr_desc(128, D, 0, 1);     // P (TMEM) x V (MN-major)
-            const uint64_t kdesc0 = smem_desc(base + SM_K, 16, 1024);       // + byte offset >> 4
+            const uint64_t qdesc0 = smem_desc(base + SM_Q, 16, 1024);       // + byte offset >> 4
+            const uint64_t kdesc0 = smem_desc(base + SM_K, 16, 1024);
             const uint64_t vdesc0 = smem_desc(base + SM_V, 16384, 1024);
             bool ok = mbar_wait(bar(B_QFULL), 0, s_abort, a.status, 0x4);
-            fence_after();
-            // S(t) -> buffer t & 1, once the softmax threads of tile t - 2 have taken its logits out
-            auto issue_s = [&](int t, bool k_ready, bool s_free) -> bool {
+            // S(t) -> buffer t % SBUF.  The buffer's previous tenant, P(t - SBUF), is read by
+            // PV(t - SBUF), which was issued before: the tensor pipe runs its MMAs in issue order.
+            auto issue_s = [&](int t, bool k_ready) -> bool {
                 const int s = t % KSTAGES;
                 const uint32_t ph = (t / KSTAGES) & 1;
-                const int sb = t & 1;
                 if (!k_ready && !mbar_wait(bar(B_KFULL + s), ph, s_abort, a.status, 0x8)) return false;
-                if (t >= 2) {
-                    if (!s_free && !mbar_wait(bar(B_SFREE + sb), ((t - 2) >> 1) & 1, s_abort, a.status, 0x10))
-                        return false;
-                    fence_after();
-                }
+                fence_after();
                 const uint64_t kdesc = kdesc0 + ((s * TILE_BYTES) >> 4);
-                const uint32_t d_s = tmem + TS + sb * 128;
+                const uint32_t d_s = tmem + TS + (t % SBUF) * 128;
                 if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        umma_ts(d_s, tmem + TQ + ks * 8, kdesc + (((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
-                                IDESC_S, ks > 0);
-                    umma_commit(bar(B_SFULL + sb));
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
+                        umma_ss(d_s, qdesc0 + off, kdesc + off, IDESC_S, ks > 0);
+                    }
+                    umma_commit(bar(B_SFULL + t % (2 * SBUF)));
                 }
                 return true;
             };
-            if (ok) ok = issue_s(0, false, true);
-            if (ok && T > 1) ok = issue_s(1, false, true);
+            for (int t = 0; ok && t < SBUF && t < T; ++t) ok = issue_s(t, false);
             for (int t = 0; ok && t < T; ++t) {
                 const int sv = t % VSTAGES;
                 const uint32_t phv = (t / VSTAGES) & 1;
-                const int sb = t & 1;
+                const int sb6 = t % (2 * SBUF);
+                const uint32_t php = (t / (2 * SBUF)) & 1;
                 // poll the barriers of this step together: their latencies overlap
-                const int t2 = t + 2;
-                const bool k_rdy = t2 < T && mbar_try(bar(B_KFULL + t2 % KSTAGES), (t2 / KSTAGES) & 1);
-                const bool f_rdy = t2 < T && mbar_try(bar(B_SFREE + sb), (t >> 1) & 1);
+                const int t3 = t + SBUF;
+                const bool k_rdy = t3 < T && mbar_try(bar(B_KFULL + t3 % KSTAGES), (t3 / KSTAGES) & 1);
                 const bool v_rdy = mbar_try(bar(B_VFULL + sv), phv);
-                const bool p_rdy = mbar_try(bar(B_PFULL + sb), (t >> 1) & 1);
-                if (t2 < T) {
-                    // S two tiles ahead, issued while P(t) is still being made: its buffer was read
-                    // out long before, and the softmax threads need it as early as possible
-                    ok = issue_s(t2, k_rdy, f_rdy);
-                    if (!ok) break;
-                }
+                const bool p_rdy = mbar_try(bar(B_PFULL + sb6), php);
                 if (!v_rdy && !mbar_wait(bar(B_VFULL + sv), phv, s_abort, a.status, 0x20)) break;
-                if (!p_rdy && !mbar_wait(bar(B_PFULL + sb), (t >> 1) & 1, s_abort, a.status, 0x40)) break;
+                if (!p_rdy && !mbar_wait(bar(B_PFULL + sb6), php, s_abort, a.status, 0x40)) break;
                 fence_after();
                 const uint64_t vdesc = vdesc0 + ((sv * TILE_BYTES) >> 4);
+                const uint32_t pb = tmem + TS + (t % SBUF) * 128;   // P(t): 32 columns at the head of each 64-column half
                 if (elect_one()) {
 #pragma unroll
                     for (int ks = 0; ks < KT / 16; ++ks)
-                        umma_ts(tmem + TO, tmem + TP + ks * 8, vdesc + ((ks * 2048) >> 4), IDESC_O, (t > 0 || ks > 0));
-                    umma_commit(bar(B_PFREE + sb));
+                        umma_ts(tmem + TO, pb + (ks >> 2) * 64 + (ks & 3) * 8, vdesc + ((ks * 2048) >> 4), IDESC_O,
+                                (t > 0 || ks > 0));
+                    umma_commit(bar(B_VEMPTY + sv));
                     if (t == T - 1) umma_commit(bar(B_OFULL));
                 }
+                __syncwarp();
+                if (t3 < T) ok = issue_s(t3, k_rdy);
             }
         }
     } else if (T > 0) {
@@ -309,15 +298,14 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
         uint64_t nref2 = 0;
         const uint64_t c2 = pack_f32x2(c, c);
         bool ok = true;
-        const uint32_t sbase = lane_base + TS + tp * 128 + hb * 64;
-        const uint32_t pbase = lane_base + TP + hb * 32;
-        const bool releaser = hb == 0 && (warp & 3) == 0 && lane == 0;   // hands stages back
+        const bool releaser = hb == 0 && (warp & 3) == 0 && lane == 0;   // hands K stages back
         for (int t = tp; t < T; t += 2) {
             const int slot = 2 * t + hb;
             const int e = slot < nU ? s_list[slot] : 0;
             const bool mine = (e >> side) & 1;
             const int nv = N - (e >> 2) * USV_BLOCK;   // keys of the block with index < N
-            if (!mbar_wait(bar(B_SFULL + tp), (t >> 1) & 1, s_abort, a.status, 0x80)) { ok = false; break; }
+            const uint32_t sbase = lane_base + TS + (t % SBUF) * 128 + hb * 64;
+            if (!mbar_wait(bar(B_SFULL + t % (2 * SBUF)), (t / (2 * SBUF)) & 1, s_abort, a.status, 0x80)) { ok = false; break; }
             fence_after();
             if (releaser) mbar_arrive(bar(B_KEMPTY + t % KSTAGES));   // S(t) is complete
             if (!have_ref && slot >= sref) {
@@ -344,42 +332,31 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                 nref2 = pack_f32x2(nref, nref);
                 have_ref = true;
             }
-            // Half of the 64 logit columns at a time, to stay within the register budget; the S
-            // buffer is handed back as soon as the second half is in registers.
+            // The weights (bf16 pairs) go back into the columns their logits came from: P(t) takes
+            // the first 32 of the 64 columns, each half written once its logits are in registers.
             uint32_t pk0[16], pk1[16];
-            {
+            if (mine) {
                 uint32_t sx[32];
-                if (mine) {
-                    tmem_ld32(sbase, sx);
-                    tmem_wait_ld();
-                    if (nv >= USV_BLOCK) weights32<false>(sx, pk0, c2, nref2, 0, nv, lr2);
-                    else weights32<true>(sx, pk0, c2, nref2, 0, nv, lr2);
-                    tmem_ld32(sbase + 32, sx);
-                }
+                tmem_ld32(sbase, sx);
                 tmem_wait_ld();
-                fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(B_SFREE + tp));
-                if (mine) {
-                    if (nv >= USV_BLOCK) weights32<false>(sx, pk1, c2, nref2, 32, nv, lr2);
-                    else weights32<true>(sx, pk1, c2, nref2, 32, nv, lr2);
-                } else {
+                if (nv >= USV_BLOCK) weights32<false>(sx, pk0, c2, nref2, 0, nv, lr2);
+                else weights32<true>(sx, pk0, c2, nref2, 0, nv, lr2);
+                tmem_ld32(sbase + 32, sx);
+                tmem_wait_ld();
+                tmem_st16(sbase, pk0);
+                if (nv >= USV_BLOCK) weights32<false>(sx, pk1, c2, nref2, 32, nv, lr2);
+                else weights32<true>(sx, pk1, c2, nref2, 32, nv, lr2);
+                tmem_st16(sbase + 16, pk1);
+            } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) pk0[j] = pk1[j] = 0u;
-                }
+                for (int j = 0; j < 16; ++j) pk0[j] = 0u;
+                tmem_st16(sbase, pk0);
+                tmem_st16(sbase + 16, pk0);
             }
-            if (t > 0) {
-                // the P buffer is free once PV(t - 1) has read it; that also frees its V stage
-                if (!mbar_wait(bar(B_PFREE + (tp ^ 1)), ((t - 1) >> 1) & 1, s_abort, a.status, 0x100)) { ok = false; break; }
-                fence_after();
-                if (releaser) mbar_arrive(bar(B_VEMPTY + (t - 1) % VSTAGES));
-            }
-            tmem_st16(pbase, pk0);
-            tmem_st16(pbase + 16, pk1);
             tmem_wait_st();
             fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B_PFULL + tp));
+            if (lane == 0) mbar_arrive(bar(B_PFULL + t % (2 * SBUF)));
         }
         // ---- epilogue
         if (ok) ok = mbar_wait(bar(B_OFULL), 0, s_abort, a.status, 0x200);
@@ -480,6 +457,7 @@ bool attn_pair_supported(const AttnArgs& a, int d) {
 int launch_attn_pair(const AttnArgs& a, int d, cudaStream_t st) {
     pr::Maps maps;
     int rc;
+    if ((rc = t5::make_bhnd_map(&maps.q, a.q, a.sq, a.B, a.H, a.N, d, "q")) != USV_OK) return rc;
     if ((rc = t5::make_bhnd_map(&maps.k, a.k, a.sk, a.B, a.H, a.N, d, "k")) != USV_OK) return rc;
     if ((rc = t5::make_bhnd_map(&maps.v, a.v, a.sv, a.B, a.H, a.N, d, "v")) != USV_OK) return rc;
     const int64_t grid = (int64_t)a.B * a.H * ((a.NB + 1) / 2);
