@@ -37,7 +37,7 @@ PAPER_CONTEXT = ("paper: 83.3x DiT-denoising / 22.7x end-to-end speedup vs dense
 # DRAM bytes per launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum)
 # from the ncu capture summarised under profiles/; a workload is listed only while its capture
 # is of the kernel as it stands (the roofline object then reports null).
-ATTN_DRAM_TRAFFIC = {}
+ATTN_DRAM_TRAFFIC = {"wan1.3b_480p": 375.4e6}
 
 
 def load_peaks():
