@@ -411,17 +411,50 @@ __global__ void __launch_bounds__(256) merge_kernel(Part p, int N, int C, int nU
     // G 16-byte chunks per lane at a time: the loads of one row are all in flight together, and
     // rows are added in ascending source index (fp32)
     constexpr int G = 3;
+    // The destination row and the first two source rows (most destinations have no more) are
+    // requested together, before any of them is used.
+    const int i0 = len <= 32 ? __shfl_sync(0xffffffffu, myid, 0) : list[0];
+    const int i1 = len < 2 ? 0 : (len <= 32 ? __shfl_sync(0xffffffffu, myid, 1) : list[1]);
+    const uint4* src0 = reinterpret_cast<const uint4*>(xb + (int64_t)i0 * C);
+    const uint4* src1 = reinterpret_cast<const uint4*>(xb + (int64_t)i1 * C);
     for (int c0 = 0; c0 < nvec; c0 += 32 * G) {
         float acc[G][8];
-        uint4 v[G];
+        uint4 v[G], va[G], vb[G];
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             const int c = c0 + g * 32 + lane;
             v[g] = c < nvec ? __ldg(srcj + c) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
-        for (int g = 0; g < G; ++g) bf16x8_to_float(v[g], acc[g]);
-        for (int s = 0; s < len; ++s) {
+        for (int g = 0; g < G; ++g) {
+            const int c = c0 + g * 32 + lane;
+            va[g] = c < nvec ? __ldg(src0 + c) : make_uint4(0, 0, 0, 0);
+        }
+        if (len >= 2) {
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const int c = c0 + g * 32 + lane;
+                vb[g] = c < nvec ? __ldg(src1 + c) : make_uint4(0, 0, 0, 0);
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            bf16x8_to_float(v[g], acc[g]);
+            float f[8];
+            bf16x8_to_float(va[g], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[g][e] += f[e];
+        }
+        if (len >= 2) {
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float f[8];
+                bf16x8_to_float(vb[g], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g][e] += f[e];
+            }
+        }
+        for (int s = 2; s < len; ++s) {
             const int i = len <= 32 ? __shfl_sync(0xffffffffu, myid, s) : list[s];
             const uint4* srci = reinterpret_cast<const uint4*>(xb + (int64_t)i * C);
 #pragma unroll
