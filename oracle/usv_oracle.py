@@ -9,6 +9,8 @@ Function -> passage of the paper (equations numbered in order of appearance):
   dense_masked_attn / sparse_attn           : Sec. 3.2, Eq. 5
   merge_plan (+ its parts)                  : Sec. 3.3, Eq. 6-11, Eq. 14
   merge_apply / unmerge                     : Sec. 3.3, Eq. 12-13 / Eq. 15
+  cube_order / select_blocks_local          : Fig. 2 caption ("partitioned into local 3D cubes",
+                                              "local cube attention" beside the top-k cubes)
 """
 import ctypes
 import os
@@ -26,6 +28,7 @@ __all__ = [
     "block_scores", "select_blocks", "dense_masked_attn", "sparse_attn", "destination_mask",
     "merge_descriptors", "merge_match", "merge_select", "merge_positions", "merge_plan",
     "merge_apply", "unmerge", "all_query_blocks", "keep_count", "key_marginal", "entropy", "allocate",
+    "cube_order", "select_blocks_local",
 ]
 
 
@@ -334,3 +337,50 @@ def allocate(h, gamma, rho_bar, rho_min, rho_max):
     _L().usvo_allocate(_p(h), h.shape[0], ctypes.c_double(gamma), ctypes.c_double(rho_bar),
                        ctypes.c_double(rho_min), ctypes.c_double(rho_max), _p(out))
     return out
+
+
+def cube_order(grid, cube):
+    """Token order in which the tokens of one local 3D cube are consecutive (Fig. 2 caption).
+
+    grid = (T, Hh, W) in raster order, cube = (ct, ch, cw).  Cubes are taken in raster order of
+    their cube coordinates, the tokens of a cube in raster order of their offsets inside it; a
+    cube cut by the edge of the grid just holds fewer tokens (nothing is padded).  Returns
+    (perm, inv): perm[p] = raster index of the token at position p of the cube order, inv its
+    inverse.  Written as the definition: sort the tokens by (cube coordinate, offset)."""
+    T, Hh, W = (int(v) for v in grid)
+    ct, ch, cw = (int(v) for v in cube)
+    t, y, x = np.meshgrid(np.arange(T), np.arange(Hh), np.arange(W), indexing="ij")
+    t, y, x = t.ravel(), y.ravel(), x.ravel()
+    # np.lexsort: last key is the primary one
+    perm = np.lexsort((x % cw, y % ch, t % ct, x // cw, y // ch, t // ct)).astype(np.int32)
+    inv = np.empty_like(perm)
+    inv[perm] = np.arange(perm.size, dtype=np.int32)
+    return perm, inv
+
+
+def select_blocks_local(scores, k_per_head):
+    """Selection with the local branch forced in: query block I always keeps key block I (its own
+    cube), plus the k_h - 1 best of the other key blocks (ties -> lowest index); ascending, -1 tail.
+    Returns (sel int32 [B,H,NBq,kmax], gap fp64 [B,H,NBq]): gap is the relative distance of the last
+    kept and the first dropped score among the other blocks (inf when nothing is dropped or
+    nothing else is kept)."""
+    s = np.ascontiguousarray(scores, dtype=np.float64)
+    B, H, NBq, NBk = s.shape
+    kph = np.asarray(k_per_head, dtype=np.int64)
+    kmax = int(kph.max())
+    sel = np.full((B, H, NBq, kmax), -1, dtype=np.int32)
+    gap = np.full((B, H, NBq), np.inf)
+    for b in range(B):
+        for h in range(H):
+            k = int(kph[h])
+            for i in range(NBq):
+                own = i if i < NBk else None
+                others = [j for j in range(NBk) if j != own]
+                others.sort(key=lambda j: (-s[b, h, i, j], j))
+                n_other = k - 1 if own is not None else k
+                keep = others[:n_other] + ([own] if own is not None else [])
+                sel[b, h, i, :k] = sorted(keep)
+                if 0 < n_other < len(others):
+                    a_, b_ = s[b, h, i, others[n_other - 1]], s[b, h, i, others[n_other]]
+                    gap[b, h, i] = (a_ - b_) / max(abs(a_), abs(b_), 1e-30)
+    return sel, gap
