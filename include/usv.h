@@ -213,6 +213,30 @@ int usv_attn_entropy(int B, int H, int N, int d, const void* q, const usv_stride
 int usv_allocate_sparsity(int L, const float* entropy, float gamma, float rho_bar, float rho_min,
                           float rho_max, float* rho);
 
+/* ------------------------------------------------------------------------------------------
+ * Local 3D cubes (overview figure, Fig. 2: queries, keys and values are "partitioned into local
+ * 3D cubes"; "local cube attention" beside the long-range "top-k cube selection").
+ *
+ * usv_cube_order: the token order in which the tokens of one cube are consecutive.  The grid is
+ * (T, Hh, W) in raster order, a cube is ct x ch x cw tokens (4 x 4 x 4 makes a cube one 64-token
+ * block).  Cubes come in raster order of their cube coordinates, the tokens of a cube in raster
+ * order of their offsets inside it; a cube cut by the edge of the grid holds fewer tokens and
+ * nothing is padded, so near the edges a 64-token block may straddle cubes.
+ *   perm: device int32 [T*Hh*W] (written), perm[p] = raster index of the token at position p.
+ *   inv : device int32 [T*Hh*W] or NULL (written), the inverse: inv[perm[p]] = p.
+ * To bring a [B,N,C] tensor into cube order call usv_token_unmerge(B, N, N, C, x, perm_b, y) with
+ * perm repeated per batch element (y[b,p] = x[b,perm[p]]); the same call with inv takes it back.
+ *
+ * usv_force_own_block: the local branch as part of the selection.  Sets scores[b,h,I,I] = +inf
+ * for I < min(NBq, NBk), in place, so that usv_select_blocks on these scores keeps, for every
+ * query block, its own block plus the k_h - 1 best of the others.
+ *   scores: device fp32 [B,H,NBq,NBk] (from usv_block_scores; modified).
+ * Both return USV_ERR_INVALID_ARG for non-positive sizes or a null pointer; nothing is launched.
+ */
+int usv_cube_order(int T, int Hh, int W, int ct, int ch, int cw, int32_t* perm, int32_t* inv,
+                   void* stream);
+int usv_force_own_block(int B, int H, int NBq, int NBk, float* scores, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -290,3 +290,35 @@ def allocate_sparsity(entropy, gamma, rho_bar, rho_min, rho_max):
                                        ctypes.c_float(rho_min), ctypes.c_float(rho_max), out),
            "usv_allocate_sparsity")
     return list(out)
+
+
+def cube_order(grid, cube=(4, 4, 4), device=None, want_inverse=True):
+    """Token order in which the tokens of one local 3D cube are consecutive: returns (perm, inv)
+    int32 [N] device tensors, perm[p] = raster index of the token at position p, inv its inverse
+    (None unless wanted)."""
+    T, Hh, W = (int(v) for v in grid)
+    ct, ch, cw = (int(v) for v in cube)
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    n = max(T * Hh * W, 1)
+    perm = torch.empty((n,), dtype=torch.int32, device=device)
+    inv = torch.empty((n,), dtype=torch.int32, device=device) if want_inverse else None
+    _check(lib().usv_cube_order(T, Hh, W, ct, ch, cw, _ptr(perm), _ptr(inv) if want_inverse else None,
+                                _stream(device)), "usv_cube_order")
+    return perm, inv
+
+
+def permute_tokens(x, index):
+    """y[b,p,:] = x[b,index[p],:] for a contiguous bf16 [B,N,C] tensor and an int32 [N] index (a
+    permutation from cube_order): a row gather through usv_token_unmerge."""
+    B = x.shape[0]
+    pos = index.unsqueeze(0).expand(B, -1).contiguous()
+    return token_unmerge(x, pos)
+
+
+def force_own_block(scores):
+    """In place: scores[b,h,I,I] = +inf, so that select_blocks keeps every query block's own block."""
+    if scores.dtype != torch.float32 or not scores.is_contiguous() or not scores.is_cuda or scores.dim() != 4:
+        raise ValueError("scores must be a contiguous CUDA fp32 [B,H,NBq,NBk] tensor")
+    B, H, NBq, NBk = scores.shape
+    _check(lib().usv_force_own_block(B, H, NBq, NBk, _ptr(scores), _stream(scores.device)), "usv_force_own_block")
+    return scores
