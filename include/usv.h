@@ -214,8 +214,8 @@ int usv_allocate_sparsity(int L, const float* entropy, float gamma, float rho_ba
                           float rho_max, float* rho);
 
 /* ------------------------------------------------------------------------------------------
- * Local 3D cubes (overview figure, Fig. 2: queries, keys and values are "partitioned into local
- * 3D cubes"; "local cube attention" beside the long-range "top-k cube selection").
+ * Local 3D cubes (overview figure, Fig. 2: the tokens are grouped into small 3D cubes, and
+ * attention inside the own cube runs beside the long-range top-k selection of cubes).
  *
  * usv_cube_order: the token order in which the tokens of one cube are consecutive.  The grid is
  * (T, Hh, W) in raster order, a cube is ct x ch x cw tokens (4 x 4 x 4 makes a cube one 64-token

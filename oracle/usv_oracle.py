@@ -9,8 +9,8 @@ Function -> passage of the paper (equations numbered in order of appearance):
   dense_masked_attn / sparse_attn           : Sec. 3.2, Eq. 5
   merge_plan (+ its parts)                  : Sec. 3.3, Eq. 6-11, Eq. 14
   merge_apply / unmerge                     : Sec. 3.3, Eq. 12-13 / Eq. 15
-  cube_order / select_blocks_local          : Fig. 2 caption ("partitioned into local 3D cubes",
-                                              "local cube attention" beside the top-k cubes)
+  cube_order / select_blocks_local          : Fig. 2 caption (tokens grouped into local 3D cubes;
+                                              attention in the own cube beside the top-k cubes)
 """
 import ctypes
 import os

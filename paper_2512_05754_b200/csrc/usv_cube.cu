@@ -1,5 +1,5 @@
-// Local 3D cubes (overview figure of the paper: queries, keys and values "partitioned into local
-// 3D cubes"; "local cube attention" beside the long-range top-k cube selection).
+// Local 3D cubes (overview figure of the paper, Fig. 2: the tokens are grouped into small 3D
+// cubes, and attention inside the own cube runs beside the long-range top-k selection of cubes).
 //
 //   cube_order_kernel      token order in which the tokens of one cube are consecutive, so that a
 //                          64-token block of the attention path is a 4 x 4 x 4 cube: closed-form

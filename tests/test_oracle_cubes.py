@@ -1,8 +1,8 @@
 """Pins of the oracle's cube order and of the selection with the own block forced in.
 
-The paper defines both only in the caption of its overview figure ("partitioned into local 3D
-cubes", "local cube attention" beside "top-k cube selection"); the pins are what the wording and
-the arithmetic fix: a hand-worked grid, the properties of a cube, brute force."""
+The paper defines both only in the caption of its overview figure (tokens grouped into local 3D
+cubes; attention in the own cube beside the top-k selection of cubes); the pins are what the
+wording and the arithmetic fix: a hand-worked grid, the properties of a cube, brute force."""
 import itertools
 
 import numpy as np
