@@ -1,9 +1,11 @@
 // Top-k key-block selection.
 //
-// Rows of up to 2048 scores (every workload here): one WARP per row, select_warp_kernel.  Each
-// lane keeps a contiguous chunk of the row as order-preserving keys in registers; the key T of
-// the k-th largest element is found bit by bit (32 warp-wide counts), then the lanes emit, in
-// ascending index, every element above T and the first (k - above) elements equal to T.
+// Rows of up to 2048 scores: one WARP per row, select_warp_kernel (with more of a row per lane
+// the register file holds too few warps: measured slower than the CTA kernel below).  The
+// row sits in registers as order-preserving keys, striped over the lanes; the key T of the k-th
+// largest element is found bit by bit (at most 32 warp-wide counts, fewer when a candidate cuts
+// the row at exactly k), then every element above T and the first (k - above) elements equal to
+// T are emitted in ascending index (two ballots per 32 elements give the positions).
 //
 // Longer rows: one CTA per row, select_kernel.
 //
@@ -121,7 +123,8 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* __rest
     for (int t = k + threadIdx.x; t < kmax; t += SEL_THREADS) out[t] = -1;
 }
 
-// One warp per row; lane l holds indices [l * KPL, (l + 1) * KPL).
+// One warp per row; lane l holds the scores of indices i * 32 + l, i < KPL (every load of the
+// row is one contiguous 128-byte line per warp).
 template <int KPL>
 __global__ void __launch_bounds__(256) select_warp_kernel(const float* __restrict__ scores,
                                                           int32_t* __restrict__ sel, int H, int NBq,
@@ -130,42 +133,51 @@ __global__ void __launch_bounds__(256) select_warp_kernel(const float* __restric
     const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (row >= rows) return;
     const int lane = threadIdx.x & 31;
+    const uint32_t lt = (1u << lane) - 1u;
     const int h = (int)((row / NBq) % H);
     const int k = heads.k[h];
     const float* src = scores + row * NBk;
     int32_t* out = sel + row * kmax;
-    const int j0 = lane * KPL;
     uint32_t key[KPL];
 #pragma unroll
-    for (int i = 0; i < KPL; ++i) key[i] = (j0 + i < NBk) ? float_key(__ldg(src + j0 + i)) : 0u;   // 0 < any real key
-    // largest T with count(key >= T) >= k, one bit at a time
+    for (int i = 0; i < KPL; ++i) key[i] = (i * 32 + lane < NBk) ? float_key(__ldg(src + i * 32 + lane)) : 0u;   // 0 < any real key
+    // Largest T with count(key >= T) >= k, one bit at a time.  As soon as a candidate leaves
+    // exactly k keys at or above it, those k are the answer and no tie can straddle the cut.
     uint32_t T = 0;
+    bool exact = false;
 #pragma unroll 1
     for (int bit = 31; bit >= 0; --bit) {
         const uint32_t cand = T | (1u << bit);
         int c = 0;
 #pragma unroll
         for (int i = 0; i < KPL; ++i) c += key[i] >= cand ? 1 : 0;
-        if (__reduce_add_sync(0xffffffffu, c) >= k) T = cand;
+        const int tot = __reduce_add_sync(0xffffffffu, c);
+        if (tot >= k) T = cand;
+        if (tot == k) { exact = true; break; }
     }
-    int ngt = 0, neq = 0;
+    // keys above the cut are kept; of the keys equal to T (the k-th largest key, when the search
+    // ran to the last bit) the lowest indices fill what is left
+    const uint32_t cut = exact ? T - 1u : T;   // kept outright: key > cut
+    int need_eq = 0;
+    if (!exact) {
+        int ngt = 0;
+#pragma unroll
+        for (int i = 0; i < KPL; ++i) ngt += key[i] > T ? 1 : 0;
+        need_eq = k - __reduce_add_sync(0xffffffffu, ngt);
+    }
+    int base = 0, eq_seen = 0;
 #pragma unroll
     for (int i = 0; i < KPL; ++i) {
-        ngt += key[i] > T ? 1 : 0;
-        neq += (key[i] == T && j0 + i < NBk) ? 1 : 0;
-    }
-    const int need_eq = k - __reduce_add_sync(0xffffffffu, ngt);   // kept among the equal ones: lowest indices
-    const int eq_before = warp_incl_scan(neq) - neq;
-    const int eq_take = min(max(need_eq - eq_before, 0), neq);
-    const int ntake = ngt + eq_take;
-    int p = warp_incl_scan(ntake) - ntake;
-    int eq_left = eq_take;
-#pragma unroll
-    for (int i = 0; i < KPL; ++i) {
-        const bool gt = key[i] > T;
-        const bool eq = key[i] == T && j0 + i < NBk && eq_left > 0;
-        if (gt || eq) out[p++] = j0 + i;
-        if (eq) --eq_left;
+        if (i * 32 < NBk) {   // uniform over the warp
+            const bool gt = key[i] > cut;
+            const bool eq = !exact && key[i] == T && i * 32 + lane < NBk;
+            const uint32_t eqb = __ballot_sync(0xffffffffu, eq);
+            const bool take = gt || (eq && eq_seen + __popc(eqb & lt) < need_eq);
+            const uint32_t tkb = __ballot_sync(0xffffffffu, take);
+            if (take) out[base + __popc(tkb & lt)] = i * 32 + lane;
+            base += __popc(tkb);
+            eq_seen += __popc(eqb);
+        }
     }
     for (int t = k + lane; t < kmax; t += 32) out[t] = -1;
 }
@@ -195,11 +207,14 @@ extern "C" int usv_select_blocks(int B, int H, int NBq, int NBk, const float* sc
     if (rows > 2147483647LL) return fail(USV_ERR_UNSUPPORTED, "select_blocks: too many rows");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const unsigned wg = (unsigned)((rows + 7) / 8);
-    if (NBk <= 512) select_warp_kernel<16><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows);
-    else if (NBk <= 1024) select_warp_kernel<32><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows);
-    else if (NBk <= 1536) select_warp_kernel<48><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows);
-    else if (NBk <= 2048) select_warp_kernel<64><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows);
+#define USV_SEL_WARP(KPL) select_warp_kernel<KPL><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows)
+    if (NBk <= 256) USV_SEL_WARP(8);
+    else if (NBk <= 512) USV_SEL_WARP(16);
+    else if (NBk <= 1024) USV_SEL_WARP(32);
+    else if (NBk <= 1536) USV_SEL_WARP(48);
+    else if (NBk <= 2048) USV_SEL_WARP(64);
     else select_kernel<<<(unsigned)rows, SEL_THREADS, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads);
+#undef USV_SEL_WARP
     USV_CHECK_LAUNCH("select_kernel");
     return USV_OK;
 }
