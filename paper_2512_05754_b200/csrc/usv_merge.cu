@@ -5,8 +5,8 @@
 //   match_kernel       Eq. 8-9   cosine of every source against every destination of its batch
 //                                element with a fused row arg-max (fp32 CUDA cores; the result
 //                                decides an integer that is compared with an fp64 evaluation)
-//   plan_kernel        Eq. 10-11, 14  radix-select of the r most confident sources, ordered
-//                                compaction, dst_of / pos
+//   plan_select_kernel Eq. 10         radix-select of the r-th most confident source
+//   plan_assign_kernel Eq. 11, 14     ordered compaction, dst_of / pos
 //   csr_* kernels      Eq. 12    sources grouped by destination
 //   merge_kernel       Eq. 13-14 warp-per-row gather + mean, 16-byte accesses
 //   unmerge_kernel     Eq. 15    warp-per-row gather copy, 16-byte accesses
@@ -185,25 +185,15 @@ __global__ void __launch_bounds__(256) match_kernel(const float* __restrict__ mh
 // ---------------------------------------------------------------------------- plan
 // One CTA (1024 threads) per batch element.  Radix-select of the r-th largest u, then an ordered
 // pass that marks the merged sources (ties to the lowest source index) and writes dst_of / pos.
-__global__ void __launch_bounds__(1024) plan_kernel(Part p, int N, int nA, int r,
-                                                    const int32_t* __restrict__ src_idx,
-                                                    const int32_t* __restrict__ jstar_s,
-                                                    const float* __restrict__ u_s,
-                                                    int32_t* __restrict__ dst_of,
-                                                    int32_t* __restrict__ pos,
-                                                    float* __restrict__ u_out,
-                                                    int32_t* __restrict__ jstar_out) {
+// Key T of the r-th most confident source and the number of sources equal to T that still merge
+// (Eq. 10 with ties to the lowest index), for 0 < r < nA.  One CTA per batch element.
+__global__ void __launch_bounds__(1024) plan_select_kernel(int nA, int r, const float* __restrict__ u_s,
+                                                           int2* __restrict__ tsel) {
     __shared__ int hist[256];
-    __shared__ int scratch[33];
     __shared__ uint32_t s_prefix;
     __shared__ int s_remaining;
     const int b = blockIdx.x;
     const float* u = u_s + (int64_t)b * nA;
-    const int32_t* js = jstar_s + (int64_t)b * nA;
-    int32_t* d_of = dst_of + (int64_t)b * N;
-    int32_t* ps = pos + (int64_t)b * N;
-    const int nU = nA - r;
-
     uint32_t T = 0xffffffffu;  // r == 0: nothing is above or equal (need_eq = 0 below)
     int need_eq = 0;
     if (r > 0) {
@@ -248,19 +238,64 @@ __global__ void __launch_bounds__(1024) plan_kernel(Part p, int N, int nA, int r
         need_eq = s_remaining;
     }
 
-    int base_eq = 0, base_un = 0;
-    for (int a0 = 0; a0 < nA; a0 += 1024) {
+    if (threadIdx.x == 0) tsel[b] = make_int2((int)T, need_eq);
+}
+
+// Sum over the CTA of one int per thread (1024 threads); `scratch` holds >= 33 ints.
+__device__ __forceinline__ int block_sum_1024(int v, int* scratch) {
+    int tot;
+    block_scan_1024(v, scratch, &tot);
+    return tot;
+}
+
+// dst_of / pos of the sources (ordered compaction of the unmerged ones, Eq. 11 and 14) and of the
+// destinations.  CTA (c, b) owns the sources [1024 c, 1024 c + 1024) of batch element b; what
+// it needs to know of the sources before its own (how many are above T, how many equal T) it
+// counts itself, so the CTAs are independent.
+__global__ void __launch_bounds__(1024) plan_assign_kernel(Part p, int N, int nA, int r, uint32_t T_imm, int need_imm,
+                                                           const int2* __restrict__ tsel,
+                                                           const int32_t* __restrict__ src_idx,
+                                                           const int32_t* __restrict__ jstar_s,
+                                                           const float* __restrict__ u_s,
+                                                           int32_t* __restrict__ dst_of,
+                                                           int32_t* __restrict__ pos,
+                                                           float* __restrict__ u_out,
+                                                           int32_t* __restrict__ jstar_out) {
+    __shared__ int scratch[33];
+    const int b = blockIdx.y;
+    const float* u = u_s + (int64_t)b * nA;
+    const int32_t* js = jstar_s + (int64_t)b * nA;
+    int32_t* d_of = dst_of + (int64_t)b * N;
+    int32_t* ps = pos + (int64_t)b * N;
+    const int nU = nA - r;
+    const uint32_t T = tsel != nullptr ? (uint32_t)tsel[b].x : T_imm;
+    const int need_eq = tsel != nullptr ? tsel[b].y : need_imm;
+    const int a0 = blockIdx.x * 1024;
+    if (a0 < nA) {
+        int gt_b = 0, eq_b = 0;
+        if (r > 0 && r < nA) {   // otherwise every source, or none, merges: ranks follow from the index
+            for (int a = threadIdx.x; a < a0; a += 1024) {
+                const uint32_t key = float_key(u[a]);
+                gt_b += key > T ? 1 : 0;
+                eq_b += key == T ? 1 : 0;
+            }
+            gt_b = block_sum_1024(gt_b, scratch);
+            eq_b = block_sum_1024(eq_b, scratch);
+        } else if (r == nA) {
+            gt_b = a0;
+        }
+        const int un_b = a0 - gt_b - min(eq_b, need_eq);   // unmerged sources before this CTA's
         const int a = a0 + threadIdx.x;
         const bool in = a < nA;
         const float ua = in ? u[a] : 0.f;
         const uint32_t key = in ? float_key(ua) : 0u;
         const int is_gt = (in && r > 0 && key > T) ? 1 : 0;
         const int is_eq = (in && r > 0 && key == T) ? 1 : 0;
-        int tot_eq, tot_un;
-        const int eq_rank = base_eq + block_scan_1024(is_eq, scratch, &tot_eq);
+        int tot;
+        const int eq_rank = eq_b + block_scan_1024(is_eq, scratch, &tot);
         const int merged = is_gt | (is_eq && eq_rank < need_eq);
         const int un = (in && !merged) ? 1 : 0;
-        const int un_rank = base_un + block_scan_1024(un, scratch, &tot_un);
+        const int un_rank = un_b + block_scan_1024(un, scratch, &tot);
         if (in) {
             const int n = src_idx[a];
             const int j = js[a];
@@ -274,10 +309,9 @@ __global__ void __launch_bounds__(1024) plan_kernel(Part p, int N, int nA, int r
             if (u_out) u_out[(int64_t)b * N + n] = ua;
             if (jstar_out) jstar_out[(int64_t)b * N + n] = j;
         }
-        base_eq += tot_eq;
-        base_un += tot_un;
     }
-    for (int o = threadIdx.x; o < p.nB; o += 1024) {
+    const int o = blockIdx.x * 1024 + threadIdx.x;
+    if (o < p.nB) {
         const int n = p.dst_token(o);
         d_of[n] = -1;
         ps[n] = nU + o;
@@ -300,25 +334,27 @@ __global__ void __launch_bounds__(256) csr_count_kernel(Part p, int N, int nU,
     else if (!p.is_dst(n)) row_src[(int64_t)b * nU + pos[(int64_t)b * N + n]] = n;
 }
 
-// exclusive scan of cnt[b,:] -> off[b,0..nB], cursor[b,:] = off[b,:nB].  One CTA per batch element.
+// exclusive scan of cnt[b,:] -> off[b,0..nB], cursor[b,:] = off[b,:nB].  CTA (c, b) owns the
+// destinations [1024 c, 1024 c + 1024) and sums the counts before its own itself.
 __global__ void __launch_bounds__(1024) csr_scan_kernel(int nB, const int32_t* __restrict__ cnt,
                                                         int32_t* __restrict__ off,
                                                         int32_t* __restrict__ cursor) {
     __shared__ int scratch[33];
-    const int b = blockIdx.x;
-    int base = 0;
-    for (int o0 = 0; o0 < nB; o0 += 1024) {
-        const int o = o0 + threadIdx.x;
-        const int c = o < nB ? cnt[(int64_t)b * nB + o] : 0;
-        int tot;
-        const int e = base + block_scan_1024(c, scratch, &tot);
-        if (o < nB) {
-            off[(int64_t)b * (nB + 1) + o] = e;
-            cursor[(int64_t)b * nB + o] = e;
-        }
-        base += tot;
+    const int b = blockIdx.y;
+    const int o0 = blockIdx.x * 1024;
+    int before = 0;
+    for (int o = threadIdx.x; o < o0; o += 1024) before += cnt[(int64_t)b * nB + o];
+    int tot;
+    block_scan_1024(before, scratch, &tot);
+    const int base = tot;
+    const int o = o0 + threadIdx.x;
+    const int c = o < nB ? cnt[(int64_t)b * nB + o] : 0;
+    const int e = base + block_scan_1024(c, scratch, &tot);
+    if (o < nB) {
+        off[(int64_t)b * (nB + 1) + o] = e;
+        cursor[(int64_t)b * nB + o] = e;
     }
-    if (threadIdx.x == 0) off[(int64_t)b * (nB + 1) + nB] = base;
+    if (o0 + 1024 >= nB && threadIdx.x == 0) off[(int64_t)b * (nB + 1) + nB] = base + tot;
 }
 
 __global__ void __launch_bounds__(256) csr_fill_kernel(Part p, int N, int r,
@@ -500,7 +536,7 @@ __global__ void __launch_bounds__(256) unmerge_kernel(int N, int Nm, int C,
 
 // ---------------------------------------------------------------------------- host side
 struct MergeWs {
-    size_t mhat, src_idx, jstar_s, u_s, row_src, cnt, off, cursor, csr, status, split, total;
+    size_t mhat, src_idx, jstar_s, u_s, row_src, cnt, off, cursor, csr, status, tsel, split, total;
 };
 
 static MergeWs merge_layout(int B, int N, int dm, int nA, int nB) {
@@ -517,6 +553,7 @@ static MergeWs merge_layout(int B, int N, int dm, int nA, int nB) {
     w.cursor = take((size_t)B * nB * 4);
     w.csr = take((size_t)B * nA * 4);
     w.status = take(256);                                       // device status word of the bounded waits
+    w.tsel = take((size_t)B * sizeof(int2));                    // selection threshold per batch element
     w.split = take(dm == 128 ? match_tc_bytes(B, N) : 0);       // bf16 hi/lo planes of the tensor-core matcher
     w.total = o;
     return w;
@@ -596,15 +633,25 @@ extern "C" int usv_token_merge(int B, int N, int C, const void* x, int Hm, int d
                 USV_CHECK_LAUNCH("match_kernel");
             }
         }
-        plan_kernel<<<B, 1024, 0, s>>>(p, N, nA, r, src_idx, jstar_s, u_s, dst_of, pos, u_out, jstar_out);
-        USV_CHECK_LAUNCH("plan_kernel");
+        const int2* tsel = nullptr;
+        if (r > 0 && r < nA) {
+            int2* tsel_w = reinterpret_cast<int2*>(base + L.tsel);
+            plan_select_kernel<<<B, 1024, 0, s>>>(nA, r, u_s, tsel_w);
+            USV_CHECK_LAUNCH("plan_select_kernel");
+            tsel = tsel_w;
+        }
+        // r = nA: every key is above 0; r = 0: no key is above or equal to the largest one
+        dim3 pg(ceil_div(nA > p.nB ? nA : p.nB, 1024), B);
+        plan_assign_kernel<<<pg, 1024, 0, s>>>(p, N, nA, r, r == nA ? 0u : 0xffffffffu, 0, tsel, src_idx, jstar_s, u_s,
+                                               dst_of, pos, u_out, jstar_out);
+        USV_CHECK_LAUNCH("plan_assign_kernel");
     }
     cudaError_t e = cudaMemsetAsync(cnt, 0, (size_t)B * p.nB * 4, s);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: memset: %s", cudaGetErrorString(e));
     dim3 tg(ceil_div(N, 256), B);
     csr_count_kernel<<<tg, 256, 0, s>>>(p, N, nU, dst_of, pos, cnt, row_src);
     USV_CHECK_LAUNCH("csr_count_kernel");
-    csr_scan_kernel<<<B, 1024, 0, s>>>(p.nB, cnt, off, cursor);
+    csr_scan_kernel<<<dim3(ceil_div(p.nB, 1024), B), 1024, 0, s>>>(p.nB, cnt, off, cursor);
     USV_CHECK_LAUNCH("csr_scan_kernel");
     if (r > 0) {
         csr_fill_kernel<<<tg, 256, 0, s>>>(p, N, r, dst_of, cursor, csr);
