@@ -9,6 +9,8 @@ Function -> passage of the paper (equations numbered in order of appearance):
   dense_masked_attn / sparse_attn           : Sec. 3.2, Eq. 5
   merge_plan (+ its parts)                  : Sec. 3.3, Eq. 6-11, Eq. 14
   merge_apply / unmerge                     : Sec. 3.3, Eq. 12-13 / Eq. 15
+  merge_match_local                         : Sec. 3.3, last paragraphs (matching kept inside
+                                              neighbouring 3D blocks), the other reading of Eq. 8-9
   cube_order / select_blocks_local          : Fig. 2 caption (tokens grouped into local 3D cubes;
                                               attention in the own cube beside the top-k cubes)
 """
@@ -28,7 +30,7 @@ __all__ = [
     "block_scores", "select_blocks", "dense_masked_attn", "sparse_attn", "destination_mask",
     "merge_descriptors", "merge_match", "merge_select", "merge_positions", "merge_plan",
     "merge_apply", "unmerge", "all_query_blocks", "keep_count", "key_marginal", "entropy", "allocate",
-    "cube_order", "select_blocks_local",
+    "cube_order", "select_blocks_local", "merge_match_local",
 ]
 
 
@@ -384,3 +386,46 @@ def select_blocks_local(scores, k_per_head):
                     a_, b_ = s[b, h, i, others[n_other - 1]], s[b, h, i, others[n_other]]
                     gap[b, h, i] = (a_ - b_) / max(abs(a_), abs(b_), 1e-30)
     return sel, gap
+
+
+def merge_match_local(mhat, grid, part, window):
+    """Best destination of every source among the destinations of nearby partition blocks only
+    (Sec. 3.3: sources and destinations confined to local 3D blocks; Eq. 8-9 with the arg-max
+    over the blocks within `window` = (wt, wh, ww) blocks of the source's own block, per axis).
+
+    The destination of a block is its first token in raster order.  Ties go to the lowest
+    destination index.  Returns (src_list int32 [n,2] of (b,i), jstar int32 [n], u fp64 [n],
+    u2 fp64 [n] = second-best similarity, -inf when there is no second candidate)."""
+    mhat = np.ascontiguousarray(mhat, dtype=np.float64)
+    B, N, dm = mhat.shape
+    T, Hh, W = (int(v) for v in grid)
+    st, sh, sw = (int(v) for v in part)
+    wt, wh, ww = (int(v) for v in window)
+    assert T * Hh * W == N and min(wt, wh, ww) >= 0
+    nbt, nby, nbx = -(-T // st), -(-Hh // sh), -(-W // sw)
+    src = np.nonzero(~destination_mask(grid, part))[0].astype(np.int32)
+    t, rem = np.divmod(src, Hh * W)
+    y, x = np.divmod(rem, W)
+    bt, by, bx = t // st, y // sh, x // sw
+    n = src.size
+    jstar = np.full((B, n), -1, dtype=np.int32)
+    u = np.full((B, n), -np.inf)
+    u2 = np.full((B, n), -np.inf)
+    # offsets in ascending order of the destination's raster index: a later candidate replaces
+    # the best one only when strictly better
+    for dt in range(-wt, wt + 1):
+        for dy in range(-wh, wh + 1):
+            for dx in range(-ww, ww + 1):
+                ct, cy, cx = bt + dt, by + dy, bx + dx
+                ok = (ct >= 0) & (ct < nbt) & (cy >= 0) & (cy < nby) & (cx >= 0) & (cx < nbx)
+                j = ((ct * st) * Hh + cy * sh) * W + cx * sw
+                w = np.nonzero(ok)[0]
+                for b in range(B):
+                    c = np.einsum("nd,nd->n", mhat[b, src[w]], mhat[b, j[w]])
+                    better = c > u[b, w]
+                    # the old best becomes the runner-up where it is beaten; otherwise c competes for runner-up
+                    u2[b, w] = np.where(better, u[b, w], np.maximum(u2[b, w], c))
+                    jstar[b, w] = np.where(better, j[w], jstar[b, w])
+                    u[b, w] = np.where(better, c, u[b, w])
+    sl = np.stack([np.repeat(np.arange(B, dtype=np.int32), n), np.tile(src, B)], axis=1)
+    return sl, jstar.reshape(-1), u.reshape(-1), u2.reshape(-1)

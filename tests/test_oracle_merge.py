@@ -181,3 +181,53 @@ def test_hand_worked_merge_example():
     assert np.allclose(y[0, :, 0], vals["merged"], rtol=1e-13)
     back = oracle.bf16_to_f64(oracle.unmerge(oracle.round_to_bf16(y), plan["pos"]))
     assert np.allclose(back[0, :, 0], vals["unmerged"], rtol=1e-13)
+
+
+# ---------------------------------------------------------------- matching inside nearby blocks
+def _unit_descriptors(B, N, dm, seed):
+    rng = np.random.default_rng(seed)
+    m = rng.standard_normal((B, N, dm))
+    return m / np.linalg.norm(m, axis=-1, keepdims=True)
+
+
+def test_local_matching_with_a_window_over_the_whole_grid_is_the_global_matching():
+    grid, part = (4, 6, 8), (2, 2, 2)
+    mhat = _unit_descriptors(2, 4 * 6 * 8, 16, 1)
+    sl_g, j_g, u_g, _ = oracle.merge_match(mhat, grid, part)
+    sl_l, j_l, u_l, _ = oracle.merge_match_local(mhat, grid, part, (2, 3, 4))
+    assert np.array_equal(sl_g, sl_l) and np.array_equal(j_g, j_l)
+    assert np.allclose(u_g, u_l, rtol=0, atol=1e-14)
+
+
+def test_local_matching_with_window_zero_picks_the_own_block():
+    grid, part = (3, 5, 7), (2, 2, 3)
+    mhat = _unit_descriptors(1, 3 * 5 * 7, 8, 2)
+    sl, j, u, u2 = oracle.merge_match_local(mhat, grid, part, (0, 0, 0))
+    i = sl[:, 1]
+    t, rem = np.divmod(i, 5 * 7)
+    y, x = np.divmod(rem, 7)
+    own = ((t // 2 * 2) * 5 + y // 2 * 2) * 7 + x // 3 * 3
+    assert np.array_equal(j, own)
+    assert np.allclose(u, np.einsum("nd,nd->n", mhat[0, i], mhat[0, own]))
+    assert np.all(np.isneginf(u2))
+
+
+def test_local_matching_brute_force():
+    grid, part, win = (3, 4, 6), (1, 2, 2), (1, 0, 1)
+    T, Hh, W = grid
+    mhat = _unit_descriptors(1, T * Hh * W, 8, 3)
+    mhat[0, 7] = mhat[0, 1]          # a duplicated direction: exact tie between two destinations' scores
+    is_dst = oracle.destination_mask(grid, part)
+    sl, j, u, u2 = oracle.merge_match_local(mhat, grid, part, win)
+    for (_, i), jj, uu, uu2 in zip(sl, j, u, u2):
+        ti, yi, xi = i // (Hh * W), (i // W) % Hh, i % W
+        cands = []
+        for d in np.nonzero(is_dst)[0]:
+            td, yd, xd = d // (Hh * W), (d // W) % Hh, d % W
+            if (abs(td // 1 - ti // 1) <= win[0] and abs(yd // 2 - yi // 2) <= win[1]
+                    and abs(xd // 2 - xi // 2) <= win[2]):
+                cands.append((-float(mhat[0, i] @ mhat[0, d]), int(d)))
+        cands.sort()
+        assert jj == cands[0][1] and abs(uu + cands[0][0]) < 1e-14
+        if len(cands) > 1:
+            assert abs(uu2 + cands[1][0]) < 1e-14
