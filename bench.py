@@ -145,12 +145,13 @@ def run_usv(args, wl, rank, world, device):
     N = inp["N"]
     dense_f, eff_f = flops(wl, N, kph)
     merging = wl.merge_part is not None
+    win = tuple(int(v) for v in args.merge_window.split(",")) if (merging and args.merge_window) else None
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
     if merging:
         # projection of the merged hidden states is harness work (outside the library); it is
         # done once, untimed, so that the timed step holds only the library's kernels.
-        zm, plan = usv.token_merge(inp["z"], inp["metric"], wl.grid, wl.merge_part, wl.r)
+        zm, plan = usv.token_merge(inp["z"], inp["metric"], wl.grid, wl.merge_part, wl.r, window=win)
         qkv = (zm @ inp["w"]).reshape(wl.B, N, 3, wl.H, wl.d)
         q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))   # [B,H,N,d] views
         o = torch.empty((wl.B, N, wl.H, wl.d), dtype=torch.bfloat16, device=device).permute(0, 2, 1, 3)
@@ -164,7 +165,7 @@ def run_usv(args, wl, rank, world, device):
         e = [ev() for _ in range(6)] if record else None
         if record: e[0].record()
         if merging:
-            usv.token_merge(inp["z"], inp["metric"], wl.grid, wl.merge_part, wl.r)
+            usv.token_merge(inp["z"], inp["metric"], wl.grid, wl.merge_part, wl.r, window=win)
         if record: e[1].record()
         s = usv.block_scores(q, k, N, N)
         if record: e[2].record()
@@ -253,7 +254,7 @@ def run_usv(args, wl, rank, world, device):
         "data": "synthetic",
         "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "d": wl.d, "N": N,
                    "blocks": (N + 63) // 64, "k_per_head": sorted(set(kph)),
-                   "merge_r": wl.r, "per_gpu": "one layer instance per GPU (heads/batch shard, no collective)",
+                   "merge_r": wl.r, "merge_window": list(win) if win else None, "per_gpu": "one layer instance per GPU (heads/batch shard, no collective)",
                    "l2": "inputs larger than L2 (q,k,v,o = %.0f MB per step), no flush" % (4 * q.numel() * 2 / 1e6)},
         "breakdown_ms": {"token_merge": float(seg_mean[0]), "block_scores": float(seg_mean[1]),
                          "select_blocks": float(seg_mean[2]), "sparse_attn_fwd": attn_ms,
@@ -357,6 +358,8 @@ def main():
     ap.add_argument("--workload", default="wan1.3b_480p")
     ap.add_argument("--impl", default="usv", choices=["usv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--merge-window", default=None,
+                    help="wt,wh,ww: keep the merge matching inside nearby partition blocks (usv arm only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "usv" else args.warmup
     wl = ui.workload(args.workload)

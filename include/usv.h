@@ -180,6 +180,18 @@ int usv_token_merge(int B, int N, int C, const void* x, int Hm, int dm, const vo
                     int32_t* pos, float* u_out, int32_t* jstar_out, void* ws, size_t ws_bytes,
                     void* stream);
 
+/* Token merge with the matching kept local (the closing paragraphs of Sec. 3.3 describe sources
+ * and destinations as confined to local 3D blocks, which Eq. 9 as printed does not): j*(i) is
+ * the best destination among the partition blocks within (wt, wh, ww) blocks of the source's
+ * own block along (t, y, x); window (0,0,0) merges every source into the destination of its own
+ * block, a window that covers the grid gives usv_token_merge.  Everything else, the workspace
+ * size included, is as for usv_token_merge.  wt, wh, ww >= 0 (else USV_ERR_INVALID_ARG).
+ */
+int usv_token_merge_local(int B, int N, int C, const void* x, int Hm, int dm, const void* metric,
+                          int T, int Hh, int W, int st, int sh, int sw, int wt, int wh, int ww,
+                          int r, void* x_merged, int32_t* dst_of, int32_t* pos, float* u_out,
+                          int32_t* jstar_out, void* ws, size_t ws_bytes, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * Token unmerge (Sec. 3.3, Eq. 15): y[b,n,:] = y_merged[b,pos[b,n],:].
  * y_merged: bf16 [B,Nm,C]; pos: int32 [B,N] with entries in [0,Nm); y: bf16 [B,N,C] (written).

@@ -210,9 +210,11 @@ class MergePlan:
     jstar: Optional[torch.Tensor] = None  # int32 [B,N]
 
 
-def token_merge(x, metric, grid, part, r, plan=None, debug=False):
+def token_merge(x, metric, grid, part, r, plan=None, debug=False, window=None):
     """Merges x [B,N,C] (bf16).  With `metric` [B,N,Hm,dm] a new plan is computed; with
-    metric=None the given `plan` is applied.  Returns (x_merged [B,N-r,C], plan)."""
+    metric=None the given `plan` is applied.  `window` = (wt, wh, ww) keeps the matching inside
+    the partition blocks that near the source's own block (None: all destinations).
+    Returns (x_merged [B,N-r,C], plan)."""
     if x.dim() != 3 or x.dtype != torch.bfloat16 or not x.is_cuda or not x.is_contiguous():
         raise ValueError("x must be a contiguous CUDA bf16 [B,N,C] tensor")
     B, N, C = x.shape
@@ -239,10 +241,17 @@ def token_merge(x, metric, grid, part, r, plan=None, debug=False):
     L = lib()
     need = L.usv_token_merge_workspace(B, N, C, Hm, dm if dm else 128)
     ws = _workspace(dev, need)
-    _check(L.usv_token_merge(B, N, C, _ptr(x), Hm, dm, _ptr(metric), T, Hh, W, st, sh, sw, int(r),
-                             _ptr(out), _ptr(plan.dst_of), _ptr(plan.pos), _ptr(u), _ptr(js),
-                             _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(dev)),
-           "usv_token_merge")
+    if window is None:
+        _check(L.usv_token_merge(B, N, C, _ptr(x), Hm, dm, _ptr(metric), T, Hh, W, st, sh, sw, int(r),
+                                 _ptr(out), _ptr(plan.dst_of), _ptr(plan.pos), _ptr(u), _ptr(js),
+                                 _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(dev)),
+               "usv_token_merge")
+    else:
+        wt, wh, ww = (int(v) for v in window)
+        _check(L.usv_token_merge_local(B, N, C, _ptr(x), Hm, dm, _ptr(metric), T, Hh, W, st, sh, sw, wt, wh, ww,
+                                       int(r), _ptr(out), _ptr(plan.dst_of), _ptr(plan.pos), _ptr(u), _ptr(js),
+                                       _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(dev)),
+               "usv_token_merge_local")
     return out, plan
 
 

@@ -371,6 +371,48 @@ __global__ void __launch_bounds__(256) csr_fill_kernel(Part p, int N, int r,
     }
 }
 
+// ---------------------------------------------------------------------------- local matching
+// The other reading of Sec. 3.3 (matching kept inside neighbouring 3D blocks): Eq. 8-9 with the
+// arg-max over the destinations of the partition blocks within (wt, wh, ww) blocks of the
+// source's own block.  One warp per source; the lanes split the descriptor, the candidates are
+// visited in ascending destination index and a later one wins only when strictly better.
+template <int DM>
+__global__ void __launch_bounds__(256) match_local_kernel(const float* __restrict__ mhat, Part p, int N, int nA,
+                                                          int wt, int wh, int ww,
+                                                          const int32_t* __restrict__ src_idx,
+                                                          int32_t* __restrict__ jstar_s, float* __restrict__ u_s) {
+    constexpr int V = DM / 32;   // floats per lane
+    const int a = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (a >= nA) return;
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const float* mb = mhat + (int64_t)b * N * DM;
+    const int i = src_idx[a];
+    const int x = i % p.W, y = (i / p.W) % p.Hh, t = i / (p.W * p.Hh);
+    const int bt = t / p.st, by = y / p.sh, bx = x / p.sw;
+    const int nBt = p.nB / (p.nHy * p.nWx);
+    float mi[V];
+#pragma unroll
+    for (int e = 0; e < V; ++e) mi[e] = mb[(int64_t)i * DM + lane * V + e];
+    float best = -INFINITY;
+    int jbest = -1;
+    for (int ct = max(bt - wt, 0); ct <= min(bt + wt, nBt - 1); ++ct)
+        for (int cy = max(by - wh, 0); cy <= min(by + wh, p.nHy - 1); ++cy)
+            for (int cx = max(bx - ww, 0); cx <= min(bx + ww, p.nWx - 1); ++cx) {
+                const int j = ((ct * p.st) * p.Hh + cy * p.sh) * p.W + cx * p.sw;
+                float c = 0.f;
+#pragma unroll
+                for (int e = 0; e < V; ++e) c = fmaf(mi[e], mb[(int64_t)j * DM + lane * V + e], c);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+                if (c > best) { best = c; jbest = j; }
+            }
+    if (lane == 0) {
+        jstar_s[(int64_t)b * nA + a] = jbest;
+        u_s[(int64_t)b * nA + a] = best;
+    }
+}
+
 // ---------------------------------------------------------------------------- merge
 // One warp per output row.  Rows [0,nU) copy an unmerged source; rows [nU, nU+nB) hold a
 // destination averaged with its merged sources, summed in ascending source index.
@@ -568,11 +610,15 @@ extern "C" size_t usv_token_merge_workspace(int B, int N, int C, int Hm, int dm)
     return usv::merge_layout(B, N, dm, N, N).total;
 }
 
-extern "C" int usv_token_merge(int B, int N, int C, const void* x, int Hm, int dm,
-                               const void* metric, int T, int Hh, int W, int st, int sh, int sw,
-                               int r, void* x_merged, int32_t* dst_of, int32_t* pos, float* u_out,
-                               int32_t* jstar_out, void* ws, size_t ws_bytes, void* stream) {
+// win: NULL = arg-max over every destination of the batch element (Eq. 8-9 as printed); else the
+// (wt, wh, ww) block window of the local reading.
+static int token_merge_impl(int B, int N, int C, const void* x, int Hm, int dm,
+                            const void* metric, int T, int Hh, int W, int st, int sh, int sw,
+                            int r, void* x_merged, int32_t* dst_of, int32_t* pos, float* u_out,
+                            int32_t* jstar_out, void* ws, size_t ws_bytes, void* stream, const int* win) {
     using namespace usv;
+    if (win != nullptr && (win[0] < 0 || win[1] < 0 || win[2] < 0))
+        return fail(USV_ERR_INVALID_ARG, "token_merge: window (%d,%d,%d) must not be negative", win[0], win[1], win[2]);
     if (B <= 0 || N <= 0 || C <= 0) return fail(USV_ERR_INVALID_ARG, "token_merge: B,N,C must be positive");
     if (T <= 0 || Hh <= 0 || W <= 0 || (int64_t)T * Hh * W != N)
         return fail(USV_ERR_INVALID_ARG, "token_merge: T*Hh*W = %lld != N = %d", (long long)T * Hh * W, N);
@@ -620,7 +666,12 @@ extern "C" int usv_token_merge(int B, int N, int C, const void* x, int Hm, int d
         if (nA > 0) {
             src_list_kernel<<<ceil_div(N, 256), 256, 0, s>>>(p, N, src_idx);
             USV_CHECK_LAUNCH("src_list_kernel");
-            if (dm == 128) {
+            if (win != nullptr) {
+                dim3 lg(ceil_div(nA, 8), B);
+                if (dm == 128) match_local_kernel<128><<<lg, 256, 0, s>>>(mhat, p, N, nA, win[0], win[1], win[2], src_idx, jstar_s, u_s);
+                else match_local_kernel<64><<<lg, 256, 0, s>>>(mhat, p, N, nA, win[0], win[1], win[2], src_idx, jstar_s, u_s);
+                USV_CHECK_LAUNCH("match_local_kernel");
+            } else if (dm == 128) {
                 // tensor cores: split-bf16 cosines (usv_match_tc.cu)
                 unsigned int* status = reinterpret_cast<unsigned int*>(base + L.status);
                 cudaError_t e0 = cudaMemsetAsync(status, 0, 4, s);
@@ -681,4 +732,22 @@ extern "C" int usv_token_unmerge(int B, int N, int Nm, int C, const void* y_merg
         static_cast<__nv_bfloat16*>(y), rows);
     USV_CHECK_LAUNCH("unmerge_kernel");
     return USV_OK;
+}
+
+extern "C" int usv_token_merge(int B, int N, int C, const void* x, int Hm, int dm,
+                               const void* metric, int T, int Hh, int W, int st, int sh, int sw,
+                               int r, void* x_merged, int32_t* dst_of, int32_t* pos, float* u_out,
+                               int32_t* jstar_out, void* ws, size_t ws_bytes, void* stream) {
+    return token_merge_impl(B, N, C, x, Hm, dm, metric, T, Hh, W, st, sh, sw, r, x_merged, dst_of, pos, u_out,
+                            jstar_out, ws, ws_bytes, stream, nullptr);
+}
+
+extern "C" int usv_token_merge_local(int B, int N, int C, const void* x, int Hm, int dm,
+                                     const void* metric, int T, int Hh, int W, int st, int sh, int sw,
+                                     int wt, int wh, int ww, int r, void* x_merged, int32_t* dst_of,
+                                     int32_t* pos, float* u_out, int32_t* jstar_out, void* ws,
+                                     size_t ws_bytes, void* stream) {
+    const int win[3] = {wt, wh, ww};
+    return token_merge_impl(B, N, C, x, Hm, dm, metric, T, Hh, W, st, sh, sw, r, x_merged, dst_of, pos, u_out,
+                            jstar_out, ws, ws_bytes, stream, win);
 }

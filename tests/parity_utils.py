@@ -72,14 +72,19 @@ def bf16_ulp_distance(a_bits, b_bits):
     return np.abs(key(a_bits) - key(b_bits))
 
 
-def check_merge_plan(plan_gpu, metric_cpu, grid, part, r, src_sample=None):
+def check_merge_plan(plan_gpu, metric_cpu, grid, part, r, src_sample=None, window=None):
     """Admissibility of a GPU merge plan against the oracle.  plan_gpu: dict of numpy arrays
     dst_of, pos, u, jstar ([B,N]).  Returns dict of counters."""
     mhat = oracle.merge_descriptors(metric_cpu)
     B, N, _ = mhat.shape
     is_dst = oracle.destination_mask(grid, part)
     src = np.nonzero(~is_dst)[0]
-    if src_sample is None:
+    if window is not None:
+        assert src_sample is None
+        sl, js, u, u2 = oracle.merge_match_local(mhat, grid, part, window)
+        sl = sl.reshape(B, -1, 2); js = js.reshape(B, -1); u = u.reshape(B, -1); u2 = u2.reshape(B, -1)
+        idx = sl[0, :, 1]
+    elif src_sample is None:
         sl, js, u, u2 = oracle.merge_match(mhat, grid, part)
         sl = sl.reshape(B, -1, 2); js = js.reshape(B, -1); u = u.reshape(B, -1); u2 = u2.reshape(B, -1)
         idx = sl[0, :, 1]
