@@ -28,6 +28,7 @@ CASES = [
     ((5, 9, 10), (2, 2, 2), (1, 2, 0), 72, 3, 128, 1, [100, 375]),     # ragged blocks, a flat window
     ((6, 20, 32), (1, 1, 2), (0, 0, 0), 128, 2, 128, 1, [1920]),        # own block only, every source merges
     ((6, 20, 32), (1, 2, 2), (1, 1, 1), 256, 4, 128, 2, [1000, 2880]),  # several launch blocks per batch element
+    ((21, 30, 52), (1, 1, 2), (1, 1, 1), 256, 12, 128, 1, [16380]),     # the Wan 480p grid and head count, every source merges
 ]
 
 
