@@ -1,32 +1,21 @@
 // Entropy-aware scheduler inputs (Sec. 3.4 of the USV paper).
 //
 //   key_marginal_kernel   Eq. 16: abar[b,j] = 1/(H N) sum_h sum_i A(h,i,j) for the block-masked
-//                         attention of Eq. 5.  One CTA per (b, h, query block): S = Q K^T per
+//                         attention of Eq. 5, d = 64 (d = 128 runs on the tensor cores,
+//                         usv_entropy_tc.cu).  One CTA per (b, h, query block): S = Q K^T per
 //                         selected key block on mma.sync, A = exp(S - lse_i) with the
 //                         log-sum-exp the attention forward wrote, column sums over the 64
 //                         rows, fp32 atomic adds into abar.
 //   entropy_kernel        Eq. 17: h[b] = -(1/log N) sum_j abar log abar.
 //   usv_allocate_sparsity Eq. 18-19 on the host: w = (1-h)^gamma, rho_l = clip(rho_bar w_l / mean w).
 //
-// This sits beside the hot path (a per-layer statistic the scheduler reads between steps), so
-// it reuses the mma.sync building blocks and the forward's LSE instead of a tcgen05 pipeline.
+// This sits beside the hot path: a per-layer statistic the scheduler reads between steps.
 #include <math.h>
 
+#include "usv_entropy.cuh"
 #include "usv_mma_sync.cuh"
 
 namespace usv {
-
-struct MargArgs {
-    const __nv_bfloat16 *q, *k;
-    usv_strides sq, sk;
-    const int32_t* sel;
-    const float* lse;     // [B,H,N] natural log of the softmax denominator (incl. the max)
-    float* marg;          // [B,N], zeroed before the launch
-    int B, H, N, NB, kmax;
-    float scale_log2;     // softmax scale * log2(e)
-    float inv_hn;         // 1 / (H N)
-    int k_per_head[USV_MAX_HEADS];
-};
 
 template <int D>
 __global__ void __launch_bounds__(128) key_marginal_kernel(const MargArgs a) {
@@ -188,15 +177,14 @@ extern "C" int usv_attn_entropy(int B, int H, int N, int d, const void* q, const
     cudaError_t e = cudaMemsetAsync(key_marginal, 0, (size_t)B * N * sizeof(float), st);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "attn_entropy: memset: %s", cudaGetErrorString(e));
     if (d == 128) {
-        const size_t smem = (size_t)3 * MmaSmem<128>::TILE * sizeof(__nv_bfloat16);
-        cudaFuncSetAttribute(key_marginal_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        key_marginal_kernel<128><<<(unsigned)grid, 128, smem, st>>>(a);
+        int rc2 = launch_marginal_tc(a, st);
+        if (rc2 != USV_OK) return rc2;
     } else {
         const size_t smem = (size_t)3 * MmaSmem<64>::TILE * sizeof(__nv_bfloat16);
         cudaFuncSetAttribute(key_marginal_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         key_marginal_kernel<64><<<(unsigned)grid, 128, smem, st>>>(a);
     }
-    USV_CHECK_LAUNCH("key_marginal_kernel");
+    if (d != 128) USV_CHECK_LAUNCH("key_marginal_kernel");
     entropy_kernel<<<B, 1024, 0, st>>>(key_marginal, N, entropy);
     USV_CHECK_LAUNCH("entropy_kernel");
     return USV_OK;
