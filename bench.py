@@ -231,6 +231,21 @@ def run_usv(args, wl, rank, world, device):
     barrier()
     e2e_ms = f0.elapsed_time(f1) / e2e_steps
 
+    entropy_ms = None
+    if args.with_entropy:
+        s_ = usv.block_scores(q, k, N, N)
+        sel_ = usv.select_blocks(s_, kph)
+        _, lse_ = usv.sparse_attn_fwd(q, k, v, sel_, kph, N=N, out=o, return_lse=True)
+        for _ in range(3):
+            usv.attn_entropy(q, k, sel_, kph, lse_, N=N)
+        g0, g1 = ev(), ev()
+        g0.record()
+        for _ in range(20):
+            usv.attn_entropy(q, k, sel_, kph, lse_, N=N)
+        g1.record()
+        torch.cuda.synchronize()
+        entropy_ms = g0.elapsed_time(g1) / 20
+
     total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, device)
     if rank != 0:
         return None
@@ -238,7 +253,17 @@ def run_usv(args, wl, rank, world, device):
     attn_ms = float(seg_mean[3])
     peak = peaks["bf16_tflops"]
     attn_eff_tflops = eff_f / (attn_ms * 1e-3) / 1e12
-    launches_per_step = 4 + (8 + 1 if merging else 0)
+    # kernels of this library per step (memsets not counted): pooling, [3-plane split, tensor-core]
+    # scores, selection, [pair overlap, pair match, pair lists, paired attention,] exact attention
+    launches_per_step = 9 if wl.d == 128 else 4
+    if merging:
+        n_dst = 1
+        for g_, p_ in zip(wl.grid, wl.merge_part):
+            n_dst *= -(-g_ // p_)
+        select = 0 if wl.r in (0, wl.N - n_dst) else 1           # the r-th largest is searched only when 0 < r < sources
+        matcher = 1 if win else (3 if wl.d == 128 else 1)          # local / split + tensor-core + rescore / SIMT
+        # descriptors, source list, matcher, [r-th largest,] plan, CSR count/scan/fill, merge; unmerge
+        launches_per_step += 2 + matcher + select + 1 + 3 + 1 + 1
     hbm = peaks["hbm_gbs"]
     pool_bytes = 2 * (wl.B * wl.H * N * wl.d * 2) + 2 * (wl.B * wl.H * ((N + 63) // 64) * wl.d * 4)
     result = {
@@ -275,6 +300,7 @@ def run_usv(args, wl, rank, world, device):
                 "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(3 * hq.numel() * 2), "d2h_bytes_per_step": int(ho.numel() * 2)},
         "gpu_launches": launches_per_step * args.steps,
+        "attn_entropy_ms": entropy_ms,
         "clocks": clocks,
         "context": PAPER_CONTEXT,
     }
@@ -358,6 +384,8 @@ def main():
     ap.add_argument("--workload", default="wan1.3b_480p")
     ap.add_argument("--impl", default="usv", choices=["usv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--with-entropy", action="store_true",
+                    help="also time usv_attn_entropy (Sec. 3.4) on the step's q, k, sel; reported beside the step")
     ap.add_argument("--merge-window", default=None,
                     help="wt,wh,ww: keep the merge matching inside nearby partition blocks (usv arm only)")
     args = ap.parse_args()
