@@ -71,6 +71,13 @@ def test_argument_validation_happens_on_the_host(L):
     assert L.usv_token_merge(1, 24, 64, p, 1, 64, p, 2, 3, 5, 1, 1, 2, 1, p, p, p, None, None, p, z, None) == 1
     assert L.usv_token_merge(1, 24, 60, p, 1, 64, p, 2, 3, 4, 1, 1, 2, 1, p, p, p, None, None, p, z, None) == 2
     assert L.usv_token_unmerge(1, 24, 30, 64, p, p, p, None) == 1
+    # local merge: a negative window; cube order: empty grid, null output; forced own block: null scores
+    assert L.usv_token_merge_local(1, 24, 64, p, 1, 64, p, 2, 3, 4, 1, 1, 2, 0, -1, 0, 3, p, p, p, None, None, p, z,
+                                   None) == 1
+    assert b"window" in L.usv_last_error()
+    assert L.usv_cube_order(0, 3, 4, 4, 4, 4, p, None, None) == 1
+    assert L.usv_cube_order(2, 3, 4, 4, 4, 4, None, None, None) == 1
+    assert L.usv_force_own_block(1, 2, 4, 4, None, None) == 1
 
 
 def test_workspace_sizes(L):
