@@ -1,7 +1,8 @@
 // Coarse stage of the key-block selection: block pooling (HBM stream) and block scores.
 //
-//   pool_kernel   : one CTA per (tensor, b, h, block); 16-byte loads, eight rows in flight per
-//                   thread, fp32 tree reduction, mean over the VALID rows of the block.
+//   pool_kernel   : one CTA per (tensor, b, h, four blocks); 16-byte loads, the next block in
+//                   flight while the current one is reduced (fp32 tree), mean over the VALID
+//                   rows of a block.
 //   scores_kernel : fp32 CUDA-core NT GEMM per (b,h), 64x64 output tile, 4x4 per thread.
 //                   Kept in fp32 (not bf16 tensor cores) because the result decides an integer
 //                   (the top-k set) that is compared with an fp64 evaluation.
@@ -18,6 +19,10 @@ struct PoolArgs {
 };
 
 // D = head dim (64 or 128).  Threads: 128.  A row of D bf16 is D/8 uint4; TPR threads per row.
+// A CTA pools POOL_SPAN consecutive blocks of one (tensor, b, h); the loads of the next block are
+// issued before the current one is reduced, so that the CTA always has a block in flight.
+constexpr int POOL_SPAN = 4;
+
 template <int D>
 __global__ void __launch_bounds__(128) pool_kernel(const PoolArgs a) {
     constexpr int TPR = D / 8;          // 16 (d=128) or 8 (d=64)
@@ -25,8 +30,9 @@ __global__ void __launch_bounds__(128) pool_kernel(const PoolArgs a) {
     constexpr int ITERS = USV_BLOCK / RPI;
     const int which = blockIdx.z;
     const int NB = a.NB[which];
-    const int I = blockIdx.x;
-    if (I >= NB) return;
+    const int I0 = blockIdx.x * POOL_SPAN;
+    if (I0 >= NB) return;
+    const int I1 = min(I0 + POOL_SPAN, NB);
     const int bh = blockIdx.y;
     const int b = bh / a.H, h = bh % a.H;
     const int N = a.N[which];
@@ -34,33 +40,43 @@ __global__ void __launch_bounds__(128) pool_kernel(const PoolArgs a) {
     const __nv_bfloat16* base =
         a.x[which] + b * a.sb[which] + h * a.sh[which] + (int64_t)col * 8;
     const int64_t sn = a.sn[which];
-    const int row0 = I * USV_BLOCK;
-    const int nvalid = min(USV_BLOCK, N - row0);
+    __shared__ float red[2][RPI][D + 4];
 
-    uint4 v[ITERS];
+    auto load_block = [&](int I, uint4* v) {
+        const int row0 = I * USV_BLOCK;
+        const int nvalid = min(USV_BLOCK, N - row0);
 #pragma unroll
-    for (int it = 0; it < ITERS; ++it) {
-        const int r = it * RPI + rg;
-        v[it] = make_uint4(0, 0, 0, 0);
-        if (r < nvalid) v[it] = __ldg(reinterpret_cast<const uint4*>(base + (row0 + r) * sn));
-    }
-    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        for (int it = 0; it < ITERS; ++it) {
+            const int r = it * RPI + rg;
+            v[it] = make_uint4(0, 0, 0, 0);
+            if (r < nvalid) v[it] = __ldg(reinterpret_cast<const uint4*>(base + (row0 + r) * sn));
+        }
+    };
+    uint4 v[ITERS], vn[ITERS];
+    load_block(I0, v);
+    for (int I = I0; I < I1; ++I) {
+        if (I + 1 < I1) load_block(I + 1, vn);
+        float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #pragma unroll
-    for (int it = 0; it < ITERS; ++it) {
-        float f[8];
-        bf16x8_to_float(v[it], f);
+        for (int it = 0; it < ITERS; ++it) {
+            float f[8];
+            bf16x8_to_float(v[it], f);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] += f[e];
-    }
-    __shared__ float red[RPI][D + 4];
+            for (int e = 0; e < 8; ++e) acc[e] += f[e];
+        }
+        float (*rd)[D + 4] = red[(I - I0) & 1];   // two buffers: one barrier per block is enough
 #pragma unroll
-    for (int e = 0; e < 8; ++e) red[rg][col * 8 + e] = acc[e];
-    __syncthreads();
-    if (threadIdx.x < D) {
-        float s = 0.f;
+        for (int e = 0; e < 8; ++e) rd[rg][col * 8 + e] = acc[e];
+        __syncthreads();
+        if (threadIdx.x < D) {
+            const int nvalid = min(USV_BLOCK, N - I * USV_BLOCK);
+            float s = 0.f;
 #pragma unroll
-        for (int g = 0; g < RPI; ++g) s += red[g][threadIdx.x];
-        a.out[which][((int64_t)bh * NB + I) * D + threadIdx.x] = s / (float)nvalid;
+            for (int g = 0; g < RPI; ++g) s += rd[g][threadIdx.x];
+            a.out[which][((int64_t)bh * NB + I) * D + threadIdx.x] = s / (float)nvalid;
+        }
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) v[it] = vn[it];
     }
 }
 
@@ -165,7 +181,7 @@ extern "C" int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void*
     a.N[0] = Nq; a.N[1] = Nk; a.NB[0] = NBq; a.NB[1] = NBk;
     a.out[0] = qbar; a.out[1] = kbar;
     a.H = H;
-    dim3 pg(NBq > NBk ? NBq : NBk, B * H, 2);
+    dim3 pg(ceil_div(NBq > NBk ? NBq : NBk, POOL_SPAN), B * H, 2);
     if (d == 128) pool_kernel<128><<<pg, 128, 0, st>>>(a);
     else pool_kernel<64><<<pg, 128, 0, st>>>(a);
     USV_CHECK_LAUNCH("pool_kernel");
@@ -248,7 +264,7 @@ extern "C" int usv_block_scores_noalloc(int B, int H, int Nq, int Nk, int d, con
     a.N[0] = Nq; a.N[1] = Nk; a.NB[0] = NBq; a.NB[1] = NBk;
     a.out[0] = qbar; a.out[1] = kbar;
     a.H = H;
-    dim3 pg(NBq > NBk ? NBq : NBk, B * H, 2);
+    dim3 pg(ceil_div(NBq > NBk ? NBq : NBk, POOL_SPAN), B * H, 2);
     if (d == 128) pool_kernel<128><<<pg, 128, 0, st>>>(a);
     else pool_kernel<64><<<pg, 128, 0, st>>>(a);
     USV_CHECK_LAUNCH("pool_kernel (noalloc)");
