@@ -289,8 +289,11 @@ int launch_scores_tc(const float* qbar, const float* kbar, float* scores, int BH
     e = cudaFuncSetAttribute(sc::scores_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sc::SMEM_BYTES);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "block_scores: smem attribute: %s", cudaGetErrorString(e));
     const int ctas = (m.NBq_pad / 128) * BH, t_all = m.NBk_pad / 128;
-    int nz = (296 + ctas - 1) / ctas;          // aim at two CTAs' worth of work per SM
+    // One CTA per SM is resident: split the key-block tiles over blockIdx.z only as far as the
+    // grid still fits one wave (148 SMs), so that no CTA pays its set-up for a single tile twice.
+    int nz = 148 / ctas;
     nz = nz < 1 ? 1 : (nz > t_all ? t_all : nz);
+    nz = (t_all + (t_all + nz - 1) / nz - 1) / ((t_all + nz - 1) / nz);   // slices that hold at least one tile
     dim3 grid(m.NBq_pad / 128, BH, nz);
     sc::scores_tc_kernel<<<grid, 192, sc::SMEM_BYTES, st>>>(m, maps);
     USV_CHECK_LAUNCH("scores_tc_kernel");
