@@ -77,7 +77,6 @@ static_assert(TS + SBUF * 128 <= TMEM_COLS, "TMEM budget");
 constexpr int NSOFT = NWG * 128;   // softmax threads
 constexpr int NTHREADS = NSOFT + 96;
 constexpr int W_TMA = NSOFT / 32, W_MMA = NSOFT / 32 + 1, W_TMA_V = NSOFT / 32 + 2;
-__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory"); }
 
 struct Maps {
     CUtensorMap q, k, v;
