@@ -81,7 +81,7 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(224, 1)
 match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -135,12 +135,13 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
             }
             __syncwarp();
         }
-    } else if (warp == 5) {
-        // ===== MMA issuer =====
+    } else if (warp == 5 || warp == 6) {
+        // ===== two MMA issuers: warp 5 takes the even tiles, warp 6 the odd ones (each tile has its
+        // own B stage and D buffer), so that one warp's barrier waits fall under the other's MMAs =====
         constexpr uint32_t IDESC = instr_desc(128, 128, 0, 0);   // A (TMEM) x B (K-major)
         const uint64_t bdesc0 = smem_desc(base + SM_B, 16, 1024);
         bool ok = mbar_wait(bar(B_AFULL), 0, s_abort, m.status, 0x20000);
-        for (int t = 0; ok && t < T; ++t) {
+        for (int t = warp - 5; ok && t < T; t += 2) {
             const int s = t % STAGES;
             const uint32_t ph = (t / STAGES) & 1;
             const int buf = t & 1;
@@ -214,11 +215,32 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(B_DFREE + buf));
                 }
-                // ascending destination order, strict improvement: equal cosines keep the lowest
+                // The chunk's maximum first, on four independent chains (a running compare over
+                // all 32 would be one long dependent chain); only a chunk that beats the best so far
+                // is searched for where.  Ascending destination order and strict improvement: equal
+                // cosines keep the lowest destination.
+                if (nvalid < 128) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float v = __uint_as_float(sr[j]);
-                    if (ch * 32 + j < nvalid && v > best) { best = v; bi = t * 128 + ch * 32 + j; }
+                    for (int j = 0; j < 32; ++j)
+                        if (ch * 32 + j >= nvalid) sr[j] = 0xff800000u;   // -inf: a destination that does not exist
+                }
+                float c0 = __uint_as_float(sr[0]), c1 = __uint_as_float(sr[1]), c2 = __uint_as_float(sr[2]),
+                      c3 = __uint_as_float(sr[3]);
+#pragma unroll
+                for (int j = 4; j < 32; j += 4) {
+                    c0 = fmaxf(c0, __uint_as_float(sr[j]));
+                    c1 = fmaxf(c1, __uint_as_float(sr[j + 1]));
+                    c2 = fmaxf(c2, __uint_as_float(sr[j + 2]));
+                    c3 = fmaxf(c3, __uint_as_float(sr[j + 3]));
+                }
+                const float cm = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
+                if (cm > best) {
+                    best = cm;
+                    int jj = 31;
+#pragma unroll
+                    for (int j = 30; j >= 0; --j)
+                        if (__uint_as_float(sr[j]) == cm) jj = j;
+                    bi = t * 128 + ch * 32 + jj;
                 }
             }
         }
@@ -299,7 +321,7 @@ int launch_match_tc(const float* mhat, const Part& p, int B, int N, int nA, cons
     cudaError_t e = cudaFuncSetAttribute(mt::match_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mt::SMEM_BYTES);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: smem attribute: %s", cudaGetErrorString(e));
     dim3 grid(m.nA_pad / 128, B);
-    mt::match_tc_kernel<<<grid, 192, mt::SMEM_BYTES, st>>>(m, maps);
+    mt::match_tc_kernel<<<grid, 224, mt::SMEM_BYTES, st>>>(m, maps);
     USV_CHECK_LAUNCH("match_tc_kernel");
     const int64_t srcs = (int64_t)B * nA;
     mt::rescore_kernel<<<(unsigned)((srcs + 7) / 8), 256, 0, st>>>(mhat, m);
