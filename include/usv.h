@@ -14,7 +14,11 @@
  *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream).
  *     Scratch memory comes from the caller (`ws`, `ws_bytes`); the matching *_workspace()
  *     function gives the size needed.  The workspace may be reused by a later call on the same
- *     stream; concurrent calls on different streams need different workspaces.
+ *     stream; concurrent calls on different streams need different workspaces.  The first
+ *     USV_WS_HEADER bytes of every workspace are a header whose first word is the device status
+ *     word: zero it once after allocating the buffer (usv_workspace_init); the entry points only
+ *     ever OR into it, so one usv_workspace_status after many calls sees a wait that gave up in
+ *     any of them.
  *   - Every function returns a usv_status.  Arguments are validated on the host before anything
  *     is launched; on a non-zero status nothing has been enqueued (USV_ERR_CUDA excepted, which
  *     reports a failed launch).  usv_last_error() gives a human-readable reason for the calling
@@ -38,6 +42,7 @@ extern "C" {
 
 #define USV_BLOCK 64
 #define USV_MAX_HEADS 128
+#define USV_WS_HEADER 256
 
 typedef enum {
     USV_OK = 0,
@@ -76,7 +81,10 @@ int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void* q, const u
 
 /* ------------------------------------------------------------------------------------------
  * usv_block_scores for callers that cannot hand over scratch memory.  (The paper has no
- * counterpart: this is a packaging variant of the entry point above, same arithmetic.)
+ * counterpart: this is a packaging variant of the entry point above.  Same definition and fp32-grade
+ * results, but not bit-identical at d = 128: this variant takes the scores from the fp32 CUDA-core
+ * kernel, usv_block_scores from the three-plane tensor-core product; the two agree to about 2e-6
+ * relative, so a top-k taken on a near-tie may resolve differently.)
  *
  * Who needs it: code that runs where device allocation is off limits -- inside a region that
  * must not call cudaMalloc (an allocator-frozen section of a host framework, a plugin
@@ -91,8 +99,10 @@ int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void* q, const u
  *     the pooled means of q and k (B*H*(NBq + NBk)*d fp32 values, each tensor rounded up to
  *     256 bytes) exceed USV_NOALLOC_SCRATCH_BYTES.
  *   - The first call on each device looks up the array's device address (a one-off, synchronous
- *     runtime query with that device current).  Make that first call before starting any
- *     stream capture on the device.
+ *     runtime query with that device current; where the runtime loads device code lazily, this
+ *     query or the first launch is also what brings the library's device image, the array
+ *     included, onto the GPU).  Make that first call before entering the region in which nothing
+ *     may be allocated, and before starting any stream capture on the device.
  *   - All calls on a device share the one array.  It keeps whatever the previous call left; every
  *     element a call reads is first written by that same call, so nothing needs clearing.  Two
  *     calls whose kernels overlap on the GPU (different streams, no ordering) race on it:
@@ -148,9 +158,22 @@ int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_str
  * Synchronises `stream`.  ws is the workspace that call used. */
 int usv_sparse_attn_fallbacks(const void* ws, void* stream, int* count);
 
-/* Reads the device status word a kernel with bounded waits leaves in its workspace.
- * Synchronises `stream`.  Returns USV_OK, USV_ERR_TIMEOUT or USV_ERR_CUDA. */
-int usv_workspace_status(const void* ws, void* stream);
+/* Zeroes the header of a freshly allocated workspace (asynchronous, on `stream`). */
+int usv_workspace_init(void* ws, void* stream);
+
+/* Reads the device status word (word 0 of the workspace header) that kernels with bounded waits
+ * OR their codes into: the tcgen05 kernels behind usv_block_scores, usv_sparse_attn_fwd,
+ * usv_token_merge and usv_attn_entropy.  Synchronises `stream`.  Returns USV_OK, USV_ERR_CUDA, or
+ * USV_ERR_TIMEOUT if any call since the last query gave up a wait (its results are then
+ * undefined); a reported word is cleared, so the next query starts afresh. */
+int usv_workspace_status(void* ws, void* stream);
+
+/* Self-test of the bounded wait (the paper has no counterpart).  Launches one warp that waits,
+ * with the same routine the kernels use but a limit of `limit_us` microseconds (1..100000), on a
+ * barrier nothing arrives at.  The wait runs out, the warp ORs 0x80000000 into the status word of
+ * `ws` and returns: usv_workspace_status(ws) then reports USV_ERR_TIMEOUT and the device context
+ * stays usable.  Nothing traps and nothing waits without a limit. */
+int usv_selftest_wait_timeout(void* ws, unsigned int limit_us, void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * Token merge (Sec. 3.3, Eq. 6-14).
@@ -211,11 +234,13 @@ int usv_token_unmerge(int B, int N, int Nm, int C, const void* y_merged, const i
  * usv_sparse_attn_fwd.  lse: fp32 [B,H,N] from that call.  key_marginal: fp32 [B,N] (written;
  * sums to 1 per batch element up to rounding).  entropy: fp32 [B] (written).  The sums use fp32
  * atomic adds: results are reproducible to rounding, not bit for bit.
+ * ws: optional device pointer to a workspace header (USV_WS_HEADER bytes are enough) whose status
+ * word receives the code of a bounded wait that gave up; NULL = not reported.
  */
 int usv_attn_entropy(int B, int H, int N, int d, const void* q, const usv_strides* sq,
                      const void* k, const usv_strides* sk, const int32_t* sel,
                      const int32_t* k_per_head, int kmax, const float* lse, float scale,
-                     float* key_marginal, float* entropy, void* stream);
+                     float* key_marginal, float* entropy, void* ws, void* stream);
 
 /* Entropy-aware allocation over the L layers of one step (Eq. 18-19), plain host arithmetic:
  *     w_l = (1 - h_l)^gamma ,   rho_l = clip(rho_min, rho_max, rho_bar * w_l / mean_l'(w_l')).

@@ -78,13 +78,21 @@ def _view(t, name):
 _ws_cache = {}
 
 
+WS_HEADER = 256
+
+
 def _workspace(device, nbytes):
-    """Grow-only scratch buffer per (device, stream)."""
+    """Grow-only scratch buffer per (device, stream).  Its header (status word) starts at zero
+    and is carried over when the buffer grows, so that workspace_status() sees every call."""
     key = (device.index, torch.cuda.current_stream(device).cuda_stream)
     buf = _ws_cache.get(key)
     if buf is None or buf.numel() < nbytes:
-        buf = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
-        _ws_cache[key] = buf
+        new = torch.empty(max(int(nbytes), WS_HEADER), dtype=torch.uint8, device=device)
+        if buf is None:
+            _check(lib().usv_workspace_init(_ptr(new), _stream(device)), "usv_workspace_init")
+        else:
+            new[:WS_HEADER].copy_(buf[:WS_HEADER])
+        _ws_cache[key] = buf = new
     return buf
 
 
@@ -148,9 +156,10 @@ def select_blocks(scores, k_per_head, kmax=None, out=None):
 
 
 def sparse_attn_fwd(q, k, v, sel, k_per_head, N=None, scale=0.0, out=None, return_f32=False,
-                    return_lse=False, impl=0):
+                    return_lse=False, impl=0, out_f32=None, out_lse=None):
     """Block-sparse attention forward.  Returns o (bf16, layout of q) and, if asked for, the
-    un-rounded fp32 output [B,H,N,d] and the log-sum-exp [B,H,N]."""
+    un-rounded fp32 output [B,H,N,d] and the log-sum-exp [B,H,N] (written into out_f32 / out_lse
+    when those contiguous fp32 tensors are given)."""
     sq, sk, sv = _view(q, "q"), _view(k, "k"), _view(v, "v")
     B, H, n, d = q.shape
     N = n if N is None else int(N)
@@ -164,8 +173,15 @@ def sparse_attn_fwd(q, k, v, sel, k_per_head, N=None, scale=0.0, out=None, retur
         else:   # token-major memory [B,N,H,d], returned as a [B,H,N,d] view
             out = torch.empty((B, n, H, d), dtype=q.dtype, device=q.device).permute(0, 2, 1, 3)
     so = _view(out, "o")
-    o32 = torch.empty((B, H, N, d), dtype=torch.float32, device=q.device) if return_f32 else None
-    lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if return_lse else None
+    o32 = lse = None
+    if return_f32:
+        o32 = torch.empty((B, H, N, d), dtype=torch.float32, device=q.device) if out_f32 is None else out_f32
+        if o32.dtype != torch.float32 or not o32.is_contiguous() or tuple(o32.shape) != (B, H, N, d):
+            raise ValueError("out_f32 must be a contiguous fp32 [B,H,N,d] tensor")
+    if return_lse:
+        lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if out_lse is None else out_lse
+        if lse.dtype != torch.float32 or not lse.is_contiguous() or tuple(lse.shape) != (B, H, N):
+            raise ValueError("out_lse must be a contiguous fp32 [B,H,N] tensor")
     L = lib()
     need = L.usv_sparse_attn_workspace(B, H, N, d, kmax)
     ws = _workspace(q.device, need)
@@ -183,16 +199,27 @@ def sparse_attn_fwd(q, k, v, sel, k_per_head, N=None, scale=0.0, out=None, retur
 
 
 def workspace_status(device=None):
-    """Synchronises and returns the device status word of the current stream's workspace."""
+    """Synchronises the current stream and returns the status (0 = ok, 5 = a bounded device-side
+    wait gave up in some call since the last query) of its workspace; a reported status is
+    cleared."""
     device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
-    ws = _workspace(device, 256)
+    ws = _workspace(device, WS_HEADER)
     return lib().usv_workspace_status(_ptr(ws), _stream(device))
+
+
+def selftest_wait_timeout(limit_us=1000, device=None):
+    """Launches the library's bounded wait on a barrier nothing arrives at; workspace_status()
+    reports USV_ERR_TIMEOUT afterwards (once)."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    ws = _workspace(device, WS_HEADER)
+    _check(lib().usv_selftest_wait_timeout(_ptr(ws), ctypes.c_uint(int(limit_us)), _stream(device)),
+           "usv_selftest_wait_timeout")
 
 
 def sparse_attn_fallbacks(device=None):
     """Query blocks of the last sparse_attn_fwd on this stream that were recomputed exactly."""
     device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
-    ws = _workspace(device, 256)
+    ws = _workspace(device, WS_HEADER)
     n = ctypes.c_int(0)
     _check(lib().usv_sparse_attn_fallbacks(_ptr(ws), _stream(device), ctypes.byref(n)),
            "usv_sparse_attn_fallbacks")
@@ -210,7 +237,7 @@ class MergePlan:
     jstar: Optional[torch.Tensor] = None  # int32 [B,N]
 
 
-def token_merge(x, metric, grid, part, r, plan=None, debug=False, window=None):
+def token_merge(x, metric, grid, part, r, plan=None, debug=False, window=None, out=None):
     """Merges x [B,N,C] (bf16).  With `metric` [B,N,Hm,dm] a new plan is computed; with
     metric=None the given `plan` is applied.  `window` = (wt, wh, ww) keeps the matching inside
     the partition blocks that near the source's own block (None: all destinations).
@@ -237,7 +264,10 @@ def token_merge(x, metric, grid, part, r, plan=None, debug=False, window=None):
             plan.u = torch.empty((B, N), dtype=torch.float32, device=dev)
             plan.jstar = torch.empty((B, N), dtype=torch.int32, device=dev)
         u, js = plan.u, plan.jstar
-    out = torch.empty((B, max(N - r, 0), C), dtype=torch.bfloat16, device=dev)
+    if out is None:
+        out = torch.empty((B, max(N - r, 0), C), dtype=torch.bfloat16, device=dev)
+    elif out.dtype != torch.bfloat16 or not out.is_contiguous() or tuple(out.shape) != (B, N - r, C):
+        raise ValueError("out must be a contiguous bf16 [B,N-r,C] tensor")
     L = lib()
     need = L.usv_token_merge_workspace(B, N, C, Hm, dm if dm else 128)
     ws = _workspace(dev, need)
@@ -283,9 +313,10 @@ def attn_entropy(q, k, sel, k_per_head, lse, N=None, scale=0.0):
     karr, _ = _k_array(k_per_head, H)
     marg = torch.empty((B, N), dtype=torch.float32, device=q.device)
     ent = torch.empty((B,), dtype=torch.float32, device=q.device)
+    ws = _workspace(q.device, WS_HEADER)
     _check(lib().usv_attn_entropy(B, H, N, d, _ptr(q), ctypes.byref(sq), _ptr(k), ctypes.byref(sk), _ptr(sel),
                                   karr, sel.shape[3], _ptr(lse), ctypes.c_float(scale), _ptr(marg), _ptr(ent),
-                                  _stream(q.device)), "usv_attn_entropy")
+                                  _ptr(ws), _stream(q.device)), "usv_attn_entropy")
     return marg, ent
 
 

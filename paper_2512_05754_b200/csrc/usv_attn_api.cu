@@ -6,13 +6,13 @@
 extern "C" size_t usv_sparse_attn_workspace(int B, int H, int N, int d, int kmax) {
     (void)d;
     if (B <= 0 || H <= 0 || N <= 0) return 0;
-    // status word + fallback counter (256-byte header), the fallback work list, the pairing plan
+    // header (status word, fallback counter), the fallback work list, the pairing plan
     const int NB = usv::ceil_div(N, USV_BLOCK);
     // sized for the worst case of every head keeping kmax blocks
     if (H > USV_MAX_HEADS) return 0;
     int32_t kk[USV_MAX_HEADS];
     for (int h = 0; h < H; ++h) kk[h] = kmax < 1 ? 1 : (kmax > NB ? NB : kmax);
-    return 256 + usv::align_up((size_t)B * H * NB * sizeof(int), 256) + usv::pair_plan_bytes(B, H, NB, kk);
+    return usv::WS_HEADER + usv::align_up((size_t)B * H * NB * sizeof(int), 256) + usv::pair_plan_bytes(B, H, NB, kk);
 }
 
 extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,
@@ -62,8 +62,8 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     a.lse = lse;
     a.status = static_cast<unsigned int*>(ws);
     a.fallback_count = reinterpret_cast<int*>(static_cast<char*>(ws) + 4);
-    a.fallback_list = reinterpret_cast<int*>(static_cast<char*>(ws) + 256);
-    void* plan_mem = static_cast<char*>(ws) + 256 + align_up((size_t)B * H * NB * sizeof(int), 256);
+    a.fallback_list = reinterpret_cast<int*>(static_cast<char*>(ws) + WS_HEADER);
+    void* plan_mem = static_cast<char*>(ws) + WS_HEADER + align_up((size_t)B * H * NB * sizeof(int), 256);
     a.pairs = nullptr;
     a.lists = nullptr;
     a.list_batch = 0;
@@ -73,7 +73,8 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     const float sc = scale == 0.f ? 1.0f / sqrtf((float)d) : scale;
     a.scale_log2 = sc * 1.4426950408889634f;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemsetAsync(ws, 0, 256, st);
+    // the status word (word 0) is sticky; everything behind it starts at zero
+    cudaError_t e = cudaMemsetAsync(static_cast<char*>(ws) + 4, 0, WS_HEADER - 4, st);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: memset: %s", cudaGetErrorString(e));
     if (impl == 0 && attn_pair_supported(a, d)) {
         int rc2 = launch_pair_plan(a, plan_mem, st);

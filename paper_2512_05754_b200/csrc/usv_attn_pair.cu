@@ -82,8 +82,9 @@ struct Maps {
     CUtensorMap q, k, v;
 };
 
-// exp2 of 32 scaled logits -> 16 packed bf16 pairs; adds the (unrounded) weights to the two
-// lanes of `acc`.  Two logits at a time on the packed-fp32 pipe.
+// exp2 of 32 scaled logits -> 16 packed bf16 pairs; adds the weights, as rounded to bf16 (what
+// the P.V product multiplies by), to the two lanes of `acc`, so that numerator and denominator of
+// a row carry the same rounding.  Two logits at a time on the packed-fp32 pipe.
 template <bool MASKED>
 __device__ __forceinline__ void weights32(const uint32_t* sr, uint32_t* pk, uint64_t c2, uint64_t nref2, int col0,
                                           int nvalid, uint64_t& acc) {
@@ -97,8 +98,8 @@ __device__ __forceinline__ void weights32(const uint32_t* sr, uint32_t* pk, uint
             if (col0 + 2 * j >= nvalid) p0 = 0.f;
             if (col0 + 2 * j + 1 >= nvalid) p1 = 0.f;
         }
-        acc = add_f32x2(acc, pack_f32x2(p0, p1));
         pk[j] = pack_bf16x2(p0, p1);
+        acc = add_f32x2(acc, pack_f32x2(__uint_as_float(pk[j] << 16), __uint_as_float(pk[j] & 0xffff0000u)));
     }
 }
 
@@ -431,14 +432,22 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
         a.fallback_list[slot] = bh_ord * NB + (threadIdx.x ? IB : IA);
     }
     if (T == 0) {
-        // no valid key block at all: defined output (zeros), as the exact kernel does
+        // no valid key block at all: defined output (zeros, log-sum-exp 0), as the exact kernel does
         __nv_bfloat16* O = a.o + b * a.so.sb + h * a.so.sh;
         for (int idx = threadIdx.x; idx < 128 * (D / 8); idx += blockDim.x) {
-            const int rr = idx / (D / 8);
+            const int rr = idx / (D / 8), cc = idx % (D / 8);
             const int Ir = rr < 64 ? IA : IB;
             const int grow = Ir * USV_BLOCK + (rr & 63);
-            if (Ir >= 0 && grow < N)
-                *reinterpret_cast<uint4*>(O + (int64_t)grow * a.so.sn + (idx % (D / 8)) * 8) = make_uint4(0, 0, 0, 0);
+            if (Ir >= 0 && grow < N) {
+                *reinterpret_cast<uint4*>(O + (int64_t)grow * a.so.sn + cc * 8) = make_uint4(0, 0, 0, 0);
+                const int64_t grow_bh = ((int64_t)b * a.H + h) * N + grow;
+                if (a.o_f32 != nullptr) {
+                    float4* o32 = reinterpret_cast<float4*>(a.o_f32 + grow_bh * D + cc * 8);
+                    o32[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    o32[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                if (a.lse != nullptr && cc == 0) a.lse[grow_bh] = 0.f;
+            }
         }
     }
     if (warp == W_MMA) {

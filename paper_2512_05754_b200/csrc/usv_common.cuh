@@ -16,6 +16,12 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Every workspace starts with a header of this many bytes.  Word 0 is the device status word:
+// kernels with bounded waits OR a code into it and nothing but usv_workspace_status /
+// usv_workspace_init ever clears it.  Word 1 counts the query blocks the attention kernel handed
+// to its exact fallback (reset by every attention call).
+constexpr size_t WS_HEADER = 256;
+
 // Validates a [B,H,N,d] view: pointer and strides 16-byte aligned, non-overlapping rows.
 int check_view(const char* name, const void* p, const usv_strides* s, int d);
 

@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(1024) entropy_kernel(const float* __restrict__
 extern "C" int usv_attn_entropy(int B, int H, int N, int d, const void* q, const usv_strides* sq,
                                 const void* k, const usv_strides* sk, const int32_t* sel,
                                 const int32_t* k_per_head, int kmax, const float* lse, float scale,
-                                float* key_marginal, float* entropy, void* stream) {
+                                float* key_marginal, float* entropy, void* ws, void* stream) {
     using namespace usv;
     if (B <= 0 || H <= 0 || N <= 0) return fail(USV_ERR_INVALID_ARG, "attn_entropy: B,H,N must be positive");
     if (d != 64 && d != 128) return fail(USV_ERR_UNSUPPORTED, "attn_entropy: d=%d (need 64 or 128)", d);
@@ -169,6 +169,7 @@ extern "C" int usv_attn_entropy(int B, int H, int N, int d, const void* q, const
     a.k = static_cast<const __nv_bfloat16*>(k);
     a.sq = *sq; a.sk = *sk;
     a.sel = sel; a.lse = lse; a.marg = key_marginal;
+    a.status = static_cast<unsigned int*>(ws);
     a.B = B; a.H = H; a.N = N; a.NB = NB; a.kmax = kmax;
     const float sc = scale == 0.f ? 1.0f / sqrtf((float)d) : scale;
     a.scale_log2 = sc * 1.4426950408889634f;

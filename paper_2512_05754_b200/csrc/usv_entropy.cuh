@@ -10,6 +10,7 @@ struct MargArgs {
     const int32_t* sel;
     const float* lse;     // [B,H,N] natural log of the softmax denominator (incl. the max)
     float* marg;          // [B,N], zeroed before the launch
+    unsigned int* status; // device status word the bounded waits report to (may be NULL)
     int B, H, N, NB, kmax;
     float scale_log2;     // softmax scale * log2(e)
     float inv_hn;         // 1 / (H N)

@@ -102,7 +102,7 @@ marginal_tc_kernel(const MargArgs a, const __grid_constant__ Maps maps) {
             n0 = (2 * t + 2 < kh) ? sel[2 * t + 2] : -1;
             n1 = (2 * t + 3 < kh) ? sel[2 * t + 3] : -1;
             const int J0 = e0 >= 0 ? e0 : 0, J1 = e1 >= 0 ? e1 : J0;
-            if (!mbar_wait(bar(B_KEMPTY + s), ph ^ 1, s_abort, nullptr, 0)) break;
+            if (!mbar_wait(bar(B_KEMPTY + s), ph ^ 1, s_abort, a.status, 0x1000000u)) break;
             const uint32_t dst = base + SM_K + s * TILE_BYTES;
             if (elect_one()) {
                 mbar_expect_tx(bar(B_KFULL + s), TILE_BYTES);
@@ -118,12 +118,12 @@ marginal_tc_kernel(const MargArgs a, const __grid_constant__ Maps maps) {
         constexpr uint32_t IDESC = instr_desc(128, USV_BLOCK, 0, 0);    // K tile (K-major) x Q (K-major)
         const uint64_t kdesc0 = smem_desc(base + SM_K, 16, 1024);
         const uint64_t qdesc0 = smem_desc(base + SM_Q, 16, 1024);
-        bool ok = mbar_wait(bar(B_QFULL), 0, s_abort, nullptr, 0);
+        bool ok = mbar_wait(bar(B_QFULL), 0, s_abort, a.status, 0x2000000u);
         for (int t = 0; ok && t < T; ++t) {
             const int s = t % KSTAGES;
             const int bf = t % NBUF;
-            if (!mbar_wait(bar(B_KFULL + s), (t / KSTAGES) & 1, s_abort, nullptr, 0)) break;
-            if (t >= NBUF && !mbar_wait(bar(B_SFREE + bf), ((t / NBUF) - 1) & 1, s_abort, nullptr, 0)) break;
+            if (!mbar_wait(bar(B_KFULL + s), (t / KSTAGES) & 1, s_abort, a.status, 0x4000000u)) break;
+            if (t >= NBUF && !mbar_wait(bar(B_SFREE + bf), ((t / NBUF) - 1) & 1, s_abort, a.status, 0x8000000u)) break;
             fence_after();
             const uint64_t kdesc = kdesc0 + ((s * TILE_BYTES) >> 4);
             if (elect_one()) {
@@ -152,7 +152,7 @@ marginal_tc_kernel(const MargArgs a, const __grid_constant__ Maps maps) {
         for (int t = 0; t < T; ++t) {
             const int bf = t % NBUF;
             const int e = (2 * t + (r >> 6) < kh) ? sel[2 * t + (r >> 6)] : -1;   // this key's block
-            if (!mbar_wait(bar(B_SFULL + bf), (t / NBUF) & 1, s_abort, nullptr, 0)) break;
+            if (!mbar_wait(bar(B_SFULL + bf), (t / NBUF) & 1, s_abort, a.status, 0x10000000u)) break;
             fence_after();
             uint32_t s0[32], s1[32];
             tmem_ld32(lane_base + bf * 64, s0);

@@ -585,6 +585,7 @@ static MergeWs merge_layout(int B, int N, int dm, int nA, int nB) {
     MergeWs w;
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    w.status = take(WS_HEADER);                                 // workspace header: word 0 = device status word
     w.mhat = take((size_t)B * N * (dm > 0 ? dm : 1) * sizeof(float));
     w.src_idx = take((size_t)nA * 4);
     w.jstar_s = take((size_t)B * nA * 4);
@@ -594,7 +595,6 @@ static MergeWs merge_layout(int B, int N, int dm, int nA, int nB) {
     w.off = take((size_t)B * (nB + 1) * 4);
     w.cursor = take((size_t)B * nB * 4);
     w.csr = take((size_t)B * nA * 4);
-    w.status = take(256);                                       // device status word of the bounded waits
     w.tsel = take((size_t)B * sizeof(int2));                    // selection threshold per batch element
     w.split = take(dm == 128 ? match_tc_bytes(B, N) : 0);       // bf16 hi/lo planes of the tensor-core matcher
     w.total = o;
@@ -674,8 +674,6 @@ static int token_merge_impl(int B, int N, int C, const void* x, int Hm, int dm,
             } else if (dm == 128) {
                 // tensor cores: split-bf16 cosines (usv_match_tc.cu)
                 unsigned int* status = reinterpret_cast<unsigned int*>(base + L.status);
-                cudaError_t e0 = cudaMemsetAsync(status, 0, 4, s);
-                if (e0 != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: memset: %s", cudaGetErrorString(e0));
                 int rc = launch_match_tc(mhat, p, B, N, nA, src_idx, jstar_s, u_s, base + L.split, status, s);
                 if (rc != USV_OK) return rc;
             } else {

@@ -144,8 +144,8 @@ __global__ void __launch_bounds__(256) scores_kernel(const float* __restrict__ q
 extern "C" size_t usv_block_scores_workspace(int B, int H, int Nq, int Nk, int d) {
     if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || d <= 0) return 0;
     const size_t nbq = usv::ceil_div(Nq, USV_BLOCK), nbk = usv::ceil_div(Nk, USV_BLOCK);
-    // pooled means of q and k; at d = 128 also the bf16 planes of the tensor-core scores kernel
-    return usv::align_up((size_t)B * H * nbq * d * sizeof(float), 256) +
+    // header, pooled means of q and k; at d = 128 also the bf16 planes of the tensor-core scores kernel
+    return usv::WS_HEADER + usv::align_up((size_t)B * H * nbq * d * sizeof(float), 256) +
            usv::align_up((size_t)B * H * nbk * d * sizeof(float), 256) +
            (d == 128 ? usv::scores_tc_bytes(B * H, (int)nbq, (int)nbk) : 0);
 }
@@ -168,8 +168,8 @@ extern "C" int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void*
         return fail(USV_ERR_WORKSPACE, "block_scores: workspace %zu < %zu", ws_bytes,
                     usv_block_scores_workspace(B, H, Nq, Nk, d));
     const int NBq = ceil_div(Nq, USV_BLOCK), NBk = ceil_div(Nk, USV_BLOCK);
-    float* qbar = static_cast<float*>(ws);
-    float* kbar = reinterpret_cast<float*>(static_cast<char*>(ws) +
+    float* qbar = reinterpret_cast<float*>(static_cast<char*>(ws) + WS_HEADER);
+    float* kbar = reinterpret_cast<float*>(static_cast<char*>(ws) + WS_HEADER +
                                            align_up((size_t)B * H * NBq * d * sizeof(float), 256));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
@@ -188,7 +188,8 @@ extern "C" int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void*
 
     if (d == 128) {
         void* mem = reinterpret_cast<char*>(kbar) + align_up((size_t)B * H * NBk * d * sizeof(float), 256);
-        return launch_scores_tc(qbar, kbar, scores, B * H, NBq, NBk, 1.0f / sqrtf((float)d), mem, st);
+        return launch_scores_tc(qbar, kbar, scores, B * H, NBq, NBk, 1.0f / sqrtf((float)d), mem,
+                                static_cast<unsigned int*>(ws), st);
     }
     dim3 sg(ceil_div(NBk, 64), ceil_div(NBq, 64), B * H);
     scores_kernel<<<sg, 256, 0, st>>>(qbar, kbar, scores, NBq, NBk, d, 1.0f / sqrtf((float)d));

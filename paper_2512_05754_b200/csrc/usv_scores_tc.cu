@@ -262,21 +262,20 @@ static int make_rows_map(CUtensorMap* map, const void* ptr, int64_t rows) {
 
 static inline int pad128(int n) { return (n + 127) / 128 * 128; }
 
-// bytes of the bf16 planes (256-byte aligned total) + 256 bytes for the status word
+// bytes of the bf16 planes (256-byte aligned total)
 size_t scores_tc_bytes(int BH, int NBq, int NBk) {
-    return 256 + align_up((size_t)BH * ((size_t)pad128(NBq) + pad128(NBk)) * sc::DM * sc::NPL * sizeof(__nv_bfloat16), 256);
+    return align_up((size_t)BH * ((size_t)pad128(NBq) + pad128(NBk)) * sc::DM * sc::NPL * sizeof(__nv_bfloat16), 256);
 }
 
 int launch_scores_tc(const float* qbar, const float* kbar, float* scores, int BH, int NBq, int NBk, float scale,
-                     void* mem, cudaStream_t st) {
+                     void* mem, unsigned int* status, cudaStream_t st) {
     sc::Args m;
     m.BH = BH; m.NBq = NBq; m.NBk = NBk; m.NBq_pad = pad128(NBq); m.NBk_pad = pad128(NBk);
     m.qbar = qbar; m.kbar = kbar; m.scores = scores; m.scale = scale;
-    m.status = static_cast<unsigned int*>(mem);
-    m.a_pl = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(mem) + 256);
+    m.status = status;
+    m.a_pl = static_cast<__nv_bfloat16*>(mem);
     m.b_pl = m.a_pl + (size_t)sc::NPL * BH * m.NBq_pad * sc::DM;
-    cudaError_t e = cudaMemsetAsync(mem, 0, 4, st);
-    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "block_scores: memset: %s", cudaGetErrorString(e));
+    cudaError_t e;
     const int64_t rows = (int64_t)BH * (m.NBq_pad + m.NBk_pad);
     sc::split3_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(m);
     USV_CHECK_LAUNCH("split3_kernel");

@@ -40,7 +40,8 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
 // its loop.  The first one to give up raises the CTA's abort flag and records `code` in the
 // device status word.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          unsigned int* status, unsigned int code) {
+                                          unsigned int* status, unsigned int code,
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
     // fast path: plain polling (each try may itself block for a short, hardware-defined time)
 #pragma unroll 1
     for (int i = 0; i < 2048; ++i)
@@ -52,7 +53,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 256; ++i)
             if (mbar_try(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (gtime() - t0 > WAIT_LIMIT_NS) {
+        if (gtime() - t0 > limit_ns) {
             *abort_flag = 1;
             if (status) atomicOr(status, code);
             return false;

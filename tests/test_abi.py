@@ -85,7 +85,8 @@ def test_workspace_sizes(L):
     L.usv_token_merge_workspace.restype = ctypes.c_size_t
     # two fp32 pooled tensors [1,12,512,128]
     means = 2 * 12 * 512 * 128 * 4                             # pooled means of q and k, fp32
-    planes = 256 + 12 * (512 + 512) * 128 * 3 * 2              # status word + three bf16 planes per operand
-    assert L.usv_block_scores_workspace(1, 12, 32760, 32760, 128) == means + planes
-    assert L.usv_block_scores_workspace(1, 2, 1024, 1024, 64) == 2 * 2 * 16 * 64 * 4   # d = 64: means only
+    planes = 12 * (512 + 512) * 128 * 3 * 2                    # three bf16 planes per operand
+    header = 256                                               # status word at the head of every workspace
+    assert L.usv_block_scores_workspace(1, 12, 32760, 32760, 128) == header + means + planes
+    assert L.usv_block_scores_workspace(1, 2, 1024, 1024, 64) == header + 2 * 2 * 16 * 64 * 4   # d = 64: header + means
     assert L.usv_token_merge_workspace(1, 32760, 1536, 12, 128) >= 32760 * 128 * 4

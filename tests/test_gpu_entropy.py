@@ -23,6 +23,9 @@ def usv():
 CASES = [
     ("tiny", 1, 2, (4, 16, 16), 64, [4, 4]),
     ("ragged_d128", 2, 3, (10, 10, 10), 128, [3, 16, 7]),
+    # several 128-key tiles per query tile of the tensor-core kernel and a partial last block
+    # (8170 = 127 blocks of 64 + 42 tokens); per-head k from one block to a quarter of them
+    ("mid_d128", 1, 4, (5, 38, 43), 128, [1, 13, 32, 7]),
 ]
 
 

@@ -128,3 +128,27 @@ def test_wan_480p_merge50(usv):
 
 def test_hunyuan_720p_mixed_keep_merge25(usv):
     _merge_pipeline(usv, ui.workload("hunyuan_720p"), 256, 48, 4)
+
+
+@pytest.mark.parametrize("pct,n_qb", [(100, 6), (25, 16), (10, 24), (5, 24)])
+def test_hunyuan_720p_uniform_keep(usv, pct, n_qb):
+    """The keep-ratio sweep of the HunyuanVideo-shaped layer run one ratio at a time (every head
+    keeps the same share of the key blocks), on the sequence left by the 25 % merge.  At keep
+    100 % every block is selected and the oracle's sparse attention IS dense softmax attention
+    (Eq. 4) over the 89 100 merged tokens."""
+    wl = ui.workload("hunyuan_720p_keep%d" % pct)
+    z = ui.make_hidden(wl, DEV)
+    w = ui.make_qkv_weight(wl, DEV)
+    metric = (z @ w[:, wl.C:2 * wl.C]).reshape(wl.B, wl.N, wl.H, wl.d).contiguous()
+    zm, plan = usv.token_merge(z, metric, wl.grid, wl.merge_part, wl.r)
+    del metric, z
+    N = wl.N_attn
+    qkv = (zm @ w).reshape(wl.B, N, 3, wl.H, wl.d)
+    q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    kph = wl.k_per_head()
+    assert kph == [(pct * wl.NB + 99) // 100] * wl.H
+    o = _attention_parity(usv, q, k, v, N, kph, n_qb, 40 + pct, check_sel=(pct != 100))
+    if pct == 100:
+        sel = usv.select_blocks(usv.block_scores(q, k, N, N), kph)
+        assert torch.equal(sel, torch.arange(wl.NB, dtype=torch.int32, device=DEV).expand_as(sel))
+    assert torch.isfinite(o[:, :, :N].float()).all()

@@ -110,11 +110,10 @@ def test_keep_all_matches_dense_attention(usv):
     qf, kf, vf = (t.double() for t in (q, k, v))
     ref = torch.softmax(qf @ kf.transpose(-1, -2) / d ** 0.5, -1) @ vf
     mx, rl2 = attn_errors(o32.cpu().numpy(), ref.numpy())
-    # White-noise values: the output is a near-cancelling average, so the 2^-9 relative rounding
-    # of the bf16 softmax weights fed to the P.V tensor-core product shows up undamped
-    # (expected relative L2 about 2^-9/sqrt(3) * sqrt(sum p^2 v^2)/|sum p v| ~ 1.1e-3..2e-3).
-    # The 1e-3 gate applies to the structured workload inputs; here 3e-3 bounds the same effect.
-    assert mx <= MAX_ABS and rl2 <= 3e-3
+    # White-noise values: the output is a near-cancelling average, the hardest case for the bf16
+    # rounding of the softmax weights fed to the P.V product.  Both kernels normalise a row by the
+    # sum of the rounded weights, which keeps it inside the stated gate.
+    assert mx <= MAX_ABS and rl2 <= REL_L2, (mx, rl2)
 
 
 @pytest.mark.parametrize("kb,expect_fallback", [(20.0, False), (64.0, True)])
@@ -138,7 +137,7 @@ def test_fixed_reference_range_and_exact_recomputation(usv, kb, expect_fallback)
     assert nfb == (4 if expect_fallback else 0)
     o_ref, lse_ref = oracle.sparse_attn(q, k, v, N, sel.numpy(), [4])
     mx, rl2 = attn_errors(o32.cpu().numpy(), o_ref.reshape(B, H, N, d))
-    assert mx <= MAX_ABS and rl2 <= 3e-3          # white-noise values: see test_keep_all_matches_dense_attention
+    assert mx <= MAX_ABS and rl2 <= REL_L2, (mx, rl2)
     assert np.abs(lse.cpu().numpy() - lse_ref.reshape(B, H, N)).max() <= 2e-3 * max(1.0, np.abs(lse_ref).max())
     assert torch.isfinite(o.float()).all()
 

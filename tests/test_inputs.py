@@ -34,6 +34,9 @@ def test_workload_table_matches_the_stated_shapes():
     h = w["hunyuan_720p"]
     assert (h.N, h.r, h.N_attn, h.NB) == (118800, 29700, 89100, 1393)
     assert h.k_per_head()[:4] == [1393, 349, 140, 70]
+    for pct, k in ((100, 1393), (25, 349), (10, 140), (5, 70)):
+        u = w["hunyuan_720p_keep%d" % pct]
+        assert (u.B, u.H, u.N_attn, u.NB, u.k_per_head()) == (2, 24, 89100, 1393, [k] * 24)
     for name, n, nb, k in (("seq_99k", 99840, 1560, 78), ("seq_131k", 131040, 2048, 103), ("seq_193k", 193440, 3023, 152)):
         assert (w[name].N, w[name].NB, w[name].k_per_head()[0]) == (n, nb, k)
 

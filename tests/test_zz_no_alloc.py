@@ -3,13 +3,16 @@
 Some hosts of this library may not allocate device memory at the point where they call it and
 have no scratch buffer to pass (an allocator-frozen section of a framework, a plugin that only
 receives tensors).  usv_block_scores_noalloc serves them from a fixed array inside the library.
-It must give exactly what usv_block_scores gives, call after call, although every call reuses the
-same array and finds the previous call's contents in it.  Collected last on purpose."""
+It must give what usv_block_scores gives (within the 2e-6 relative gate both carry against the
+oracle: at d = 128 the two run different kernels, so they are not bit-identical), call after
+call, although every call reuses the same array and finds the previous call's contents in it.
+Collected last on purpose."""
 import ctypes
 
 import pytest
 import torch
 
+import oracle
 import usv_inputs as ui
 
 
@@ -52,3 +55,7 @@ def test_noalloc_matches_block_scores_on_two_calls_in_a_row():
     assert (got_b - ref_b).abs().max().item() <= 2e-6 * max(1.0, ref_b.abs().max().item())
     assert (got_c - ref_a).abs().max().item() <= tol
     assert got_a.data_ptr() == out_a.data_ptr()
+    # and against the definition itself: the fp64 oracle on the same bytes
+    for got, (qq, kk, n) in ((got_a, (q, k, N)), (got_c, (q, k, N)), (got_b, (q2, k2, wl2.N))):
+        ref = oracle.block_scores(oracle.block_pool(qq.cpu(), n), oracle.block_pool(kk.cpu(), n))
+        assert abs(got.cpu().numpy() - ref).max() <= 2e-6 * max(1.0, abs(ref).max())

@@ -193,6 +193,16 @@ WORKLOADS = [
              note="length sweep, 131 040 tokens, 2048 blocks, keep 5%"),
     Workload("seq_193k", 7, 1, 12, 128, (31, 60, 104), (5,),
              note="length sweep, 193 440 tokens, 3023 blocks, keep 5%"),
+    # The HunyuanVideo-shaped layer with one keep ratio on every head: the four points of its
+    # keep-ratio sweep run one at a time (keep 100 % is dense attention over the merged sequence).
+    Workload("hunyuan_720p_keep100", 8, 2, 24, 128, (33, 45, 80), (100,),
+             merge_part=(1, 1, 2), merge_percent=25, note="uniform keep 100% (dense), 25% merge"),
+    Workload("hunyuan_720p_keep25", 9, 2, 24, 128, (33, 45, 80), (25,),
+             merge_part=(1, 1, 2), merge_percent=25, note="uniform keep 25%, 25% merge"),
+    Workload("hunyuan_720p_keep10", 10, 2, 24, 128, (33, 45, 80), (10,),
+             merge_part=(1, 1, 2), merge_percent=25, note="uniform keep 10%, 25% merge"),
+    Workload("hunyuan_720p_keep5", 11, 2, 24, 128, (33, 45, 80), (5,),
+             merge_part=(1, 1, 2), merge_percent=25, note="uniform keep 5%, 25% merge"),
 ]
 
 
