@@ -18,6 +18,7 @@ struct AttnArgs {
     // their work ids here; the exact kernel, launched in list mode, recomputes them.
     int* fallback_list;
     int* fallback_count;
+    int* work_counter;      // zeroed before the launch: the persistent CTAs of the tcgen05 kernel draw their items from it
     const int2* pairs;      // [B,H,ceil(NB/2)] query-block pairs of the tcgen05 kernel (head-major, not head-ordered)
     // Union key-block lists of the pairs: for (b, h, pair) at lists + b * list_batch + list_off[h] +
     // pair * list_stride(h): [0] = number of entries, then (key block << 2) | in-A | in-B << 1, ascending.

@@ -62,6 +62,7 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     a.lse = lse;
     a.status = static_cast<unsigned int*>(ws);
     a.fallback_count = reinterpret_cast<int*>(static_cast<char*>(ws) + 4);
+    a.work_counter = reinterpret_cast<int*>(static_cast<char*>(ws) + 8);
     a.fallback_list = reinterpret_cast<int*>(static_cast<char*>(ws) + WS_HEADER);
     void* plan_mem = static_cast<char*>(ws) + WS_HEADER + align_up((size_t)B * H * NB * sizeof(int), 256);
     a.pairs = nullptr;

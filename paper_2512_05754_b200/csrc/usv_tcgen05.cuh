@@ -36,6 +36,16 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
         : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     return done;
 }
+// Non-blocking test of a barrier phase (never suspends the thread, unlike try_wait).
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done;
+}
 // Bounded wait.  Returns false when it gave up (or another role already had): the caller leaves
 // its loop.  The first one to give up raises the CTA's abort flag and records `code` in the
 // device status word.
