@@ -4,8 +4,6 @@
 
 namespace usv {
 
-constexpr int PLAN_WINDOW = 64;   // pairing looks at this many query blocks on each side
-
 struct AttnArgs {
     const __nv_bfloat16 *q, *k, *v;
     __nv_bfloat16* o;
