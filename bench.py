@@ -34,10 +34,26 @@ PAPER_CONTEXT = ("paper: 83.3x DiT-denoising / 22.7x end-to-end speedup vs dense
                  "(sparsity 0.95, 3 steps vs 50) on 1x NVIDIA H20, precision unstated; "
                  "no kernel-level number is published")
 
-# DRAM bytes per launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum)
-# from the ncu capture summarised under profiles/; a workload is listed only while its capture
-# is of the kernel as it stands (the roofline object then reports null).
-ATTN_DRAM_TRAFFIC = {"wan1.3b_480p": 375.4e6}
+ATTN_KERNEL_SOURCE = os.path.join(ROOT, "paper_2512_05754_b200", "csrc", "usv_attn_pair.cu")
+ATTN_PROFILE = os.path.join(ROOT, "profiles", "attn_pair_kernel_wan480p.md")
+
+
+def attn_dram_traffic(workload):
+    """DRAM bytes per launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum)
+    from the ncu summary under profiles/, which records the sha256 prefix of the kernel source it
+    was captured on in a line `dram_traffic: workload=<name> bytes=<float> source_sha256=<16 hex>`.
+    None once the kernel source has changed since (or for a workload without a capture)."""
+    import hashlib
+    import re
+    try:
+        text = open(ATTN_PROFILE).read()
+        sha = hashlib.sha256(open(ATTN_KERNEL_SOURCE, "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+    for m in re.finditer(r"dram_traffic:\s*workload=(\S+)\s+bytes=(\S+)\s+source_sha256=([0-9a-f]{16})", text):
+        if m.group(1) == workload and m.group(3) == sha:
+            return float(m.group(2))
+    return None
 
 
 def load_peaks():
@@ -126,6 +142,18 @@ def job_value(world, flops_per_rank, ms_per_step):
     return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
 
 
+def make_config(wl, merge_window=None):
+    """The workload description both arms print (identical keys and values)."""
+    N = wl.N_attn
+    return {"workload": wl.name, "B": wl.B, "H": wl.H, "d": wl.d, "N": N, "blocks": (N + 63) // 64,
+            "k_per_head": sorted(set(wl.k_per_head())), "merge_r": wl.r,
+            "merge_window": list(merge_window) if merge_window else None,
+            "per_gpu": "one layer instance per GPU (heads/batch shard, no collective)",
+            "l2": ("inputs larger than L2 (q,k,v,o = %.0f MB per step), no flush" if 4 * wl.B * wl.H * N * wl.d * 2 > 126e6
+                   else "q,k,v,o = %.1f MB per step: fits in L2, not flushed (sanity workload)")
+                  % (4 * wl.B * wl.H * N * wl.d * 2 / 1e6)}
+
+
 def build_inputs(wl, device):
     """Device-resident inputs of one step.  Returns a dict."""
     if wl.merge_part is None:
@@ -135,6 +163,57 @@ def build_inputs(wl, device):
     w = ui.make_qkv_weight(wl, device)                               # [C,3C]
     metric = (z @ w[:, wl.C:2 * wl.C]).reshape(wl.B, wl.N, wl.H, wl.d).contiguous()
     return dict(z=z, w=w, metric=metric, N=wl.N_attn)
+
+
+def time_call(fn, iters=20, warmup=3):
+    """Mean CUDA-event time of fn() in ms (current stream)."""
+    for _ in range(warmup):
+        fn()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def hbm_entry(call, kernels, nbytes, ms, peak_gbs, note=None):
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    d = {"call": call, "kernels": kernels, "bound": "hbm", "bytes": int(nbytes), "ms": ms,
+         "achieved": gbs, "peak": peak_gbs, "unit": "GB/s", "frac": gbs / peak_gbs}
+    if note:
+        d["note"] = note
+    return d
+
+
+def merge_path_rooflines(usv, device, peak_gbs):
+    """HBM-bound calls of the merge path, timed on the 50 %-merge Wan 480p workload (hidden
+    states 100.6 MB + merged 50.3 MB per call: larger than L2, no flush): applying a stored plan
+    (CSR build + merge_kernel) and the unmerge gather."""
+    wl = ui.workload("wan1.3b_480p_merge50")
+    z = ui.make_hidden(wl, device)
+    w = ui.make_qkv_weight(wl, device)
+    metric = (z @ w[:, wl.C:2 * wl.C]).reshape(wl.B, wl.N, wl.H, wl.d).contiguous()
+    del w
+    zm, plan = usv.token_merge(z, metric, wl.grid, wl.merge_part, wl.r)
+    y = torch.empty_like(z)
+    zm2 = torch.empty_like(zm)
+    ms_plan = time_call(lambda: usv.token_merge(z, metric, wl.grid, wl.merge_part, wl.r, out=zm2))
+    ms_apply = time_call(lambda: usv.token_merge(z, None, wl.grid, wl.merge_part, wl.r, plan=plan, out=zm2))
+    ms_unm = time_call(lambda: usv.token_unmerge(zm, plan.pos, out=y))
+    moved = z.numel() * 2 + zm.numel() * 2
+    desc_bytes = metric.numel() * 2 + wl.B * wl.N * wl.d * 4
+    return [
+        hbm_entry("usv_token_merge(metric=NULL)", "csr_count/scan/fill + merge_kernel", moved, ms_apply, peak_gbs,
+                  "merge_kernel streams the bytes; the three CSR kernels before it are latency-bound"),
+        hbm_entry("usv_token_unmerge", "unmerge_kernel", moved, ms_unm, peak_gbs),
+        {"call": "usv_token_merge(metric)", "kernels": "desc + split + match_tc + rescore + plan + CSR + merge",
+         "bound": "tensor (matching) + hbm (descriptors, merge)", "ms": ms_plan,
+         "bytes_descriptors": int(desc_bytes), "bytes_merge": int(moved),
+         "note": "whole call; the plan-building part is %.4f ms" % (ms_plan - ms_apply)},
+    ], {"workload": wl.name, "B": wl.B, "N": wl.N, "C": wl.C, "r": wl.r}
 
 
 def run_usv(args, wl, rank, world, device):
@@ -194,30 +273,52 @@ def run_usv(args, wl, rank, world, device):
     t_wall0 = time.time()
     e0, e1 = ev(), ev()
     barrier()
+    launches0 = usv.kernel_launches()
     e0.record()
     for _ in range(args.steps):
         step(record=True)
     e1.record()
+    launches = usv.kernel_launches() - launches0     # the library's own count of what it enqueued
     barrier()
     t_wall1 = time.time()
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     total_ms = e0.elapsed_time(e1)
     seg = np.array([[m[i].elapsed_time(m[i + 1]) for i in range(5)] for m in marks])  # ms
     seg_mean = seg.mean(0)
-    assert usv.workspace_status() == 0
+    # the status word is sticky: a bounded wait that gave up in ANY step shows up here
+    assert usv.workspace_status() == 0, "a device-side wait gave up during the timed steps"
 
-    # ---- end to end through the public API with pinned host buffers
-    hq, hk, hv = (t.contiguous().cpu().pin_memory() for t in (q, k, v))
-    ho = torch.empty(o.shape, dtype=o.dtype).pin_memory()
-    dq, dk, dv = (torch.empty_like(t, device=device) for t in (hq, hk, hv))
-    do = torch.empty_like(dq)
+    # ---- end to end through the public API with pinned host buffers: every step copies its
+    # inputs from the host, runs the whole path and copies the result back
+    if merging:
+        hz, hm = inp["z"].cpu().pin_memory(), inp["metric"].cpu().pin_memory()
+        dz, dmet = torch.empty_like(inp["z"]), torch.empty_like(inp["metric"])
+        hy = torch.empty(inp["z"].shape, dtype=torch.bfloat16).pin_memory()
+        do = torch.empty((wl.B, N, wl.H, wl.d), dtype=torch.bfloat16, device=device).permute(0, 2, 1, 3)
+        h2d, d2h = hz.numel() * 2 + hm.numel() * 2, hy.numel() * 2
 
-    def e2e_step():
-        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
-        s = usv.block_scores(dq, dk, N, N)
-        sel = usv.select_blocks(s, kph)
-        usv.sparse_attn_fwd(dq, dk, dv, sel, kph, N=N, out=do)
-        ho.copy_(do, non_blocking=True)
+        def e2e_step():
+            dz.copy_(hz, non_blocking=True); dmet.copy_(hm, non_blocking=True)
+            zm_, plan_ = usv.token_merge(dz, dmet, wl.grid, wl.merge_part, wl.r, window=win)
+            qkv_ = (zm_ @ inp["w"]).reshape(wl.B, N, 3, wl.H, wl.d)      # harness projection (cuBLAS), inside the timed region
+            q_, k_, v_ = (qkv_[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+            sel_ = usv.select_blocks(usv.block_scores(q_, k_, N, N), kph)
+            usv.sparse_attn_fwd(q_, k_, v_, sel_, kph, N=N, out=do)
+            y_ = usv.token_unmerge(do.permute(0, 2, 1, 3).reshape(wl.B, N, wl.C), plan_.pos)
+            hy.copy_(y_, non_blocking=True)
+    else:
+        hq, hk, hv = (t.contiguous().cpu().pin_memory() for t in (q, k, v))
+        ho = torch.empty(o.shape, dtype=o.dtype).pin_memory()
+        dq, dk, dv = (torch.empty_like(t, device=device) for t in (hq, hk, hv))
+        do = torch.empty_like(dq)
+        h2d, d2h = 3 * hq.numel() * 2, ho.numel() * 2
+
+        def e2e_step():
+            dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+            s = usv.block_scores(dq, dk, N, N)
+            sel = usv.select_blocks(s, kph)
+            usv.sparse_attn_fwd(dq, dk, dv, sel, kph, N=N, out=do)
+            ho.copy_(do, non_blocking=True)
 
     e2e_steps = max(3, min(args.steps, 20))
     for _ in range(3):
@@ -230,21 +331,14 @@ def run_usv(args, wl, rank, world, device):
     f1.record()
     barrier()
     e2e_ms = f0.elapsed_time(f1) / e2e_steps
+    assert usv.workspace_status() == 0
 
     entropy_ms = None
     if args.with_entropy:
         s_ = usv.block_scores(q, k, N, N)
         sel_ = usv.select_blocks(s_, kph)
         _, lse_ = usv.sparse_attn_fwd(q, k, v, sel_, kph, N=N, out=o, return_lse=True)
-        for _ in range(3):
-            usv.attn_entropy(q, k, sel_, kph, lse_, N=N)
-        g0, g1 = ev(), ev()
-        g0.record()
-        for _ in range(20):
-            usv.attn_entropy(q, k, sel_, kph, lse_, N=N)
-        g1.record()
-        torch.cuda.synchronize()
-        entropy_ms = g0.elapsed_time(g1) / 20
+        entropy_ms = time_call(lambda: usv.attn_entropy(q, k, sel_, kph, lse_, N=N))
 
     total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, device)
     if rank != 0:
@@ -253,19 +347,20 @@ def run_usv(args, wl, rank, world, device):
     attn_ms = float(seg_mean[3])
     peak = peaks["bf16_tflops"]
     attn_eff_tflops = eff_f / (attn_ms * 1e-3) / 1e12
-    # kernels of this library per step (memsets not counted): pooling, [3-plane split, tensor-core]
-    # scores, selection, [pair overlap, pair match, pair lists, paired attention,] exact attention
-    launches_per_step = 9 if wl.d == 128 else 4
-    if merging:
-        n_dst = 1
-        for g_, p_ in zip(wl.grid, wl.merge_part):
-            n_dst *= -(-g_ // p_)
-        select = 0 if wl.r in (0, wl.N - n_dst) else 1           # the r-th largest is searched only when 0 < r < sources
-        matcher = 1 if win else (3 if wl.d == 128 else 1)          # local / split + tensor-core + rescore / SIMT
-        # descriptors, source list, matcher, [r-th largest,] plan, CSR count/scan/fill, merge; unmerge
-        launches_per_step += 2 + matcher + select + 1 + 3 + 1 + 1
     hbm = peaks["hbm_gbs"]
-    pool_bytes = 2 * (wl.B * wl.H * N * wl.d * 2) + 2 * (wl.B * wl.H * ((N + 63) // 64) * wl.d * 4)
+    NB = (N + 63) // 64
+    # algorithmic bytes: Q and K read once, fp32 means written; scores read once, selection written
+    pool_bytes = 2 * (wl.B * wl.H * N * wl.d * 2) + 2 * (wl.B * wl.H * NB * wl.d * 4)
+    scores_bytes = wl.B * wl.H * NB * NB * 4
+    select_bytes = scores_bytes + wl.B * wl.H * NB * max(kph) * 4
+    # the streaming kernel of usv_block_scores by itself (pool_kernel: first launch of the call)
+    hbm_list = [
+        hbm_entry("usv_block_scores", "pool_kernel + scores (tensor-core) kernel", pool_bytes + scores_bytes,
+                  float(seg_mean[1]), hbm,
+                  "whole call: the pooling stream plus the small score product and its launch gaps"),
+        hbm_entry("usv_select_blocks", "select kernel", select_bytes, float(seg_mean[2]), hbm,
+                  "latency-bound: one warp (rows <= 2048 scores) or CTA per row searches its k-th largest score"),
+    ]
     result = {
         "metric": "sparse_attn_dense_equiv_tflops",
         "value": job_value(world, dense_f, ms_step),
@@ -277,37 +372,45 @@ def run_usv(args, wl, rank, world, device):
         "vs_baseline": None,
         "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "d": wl.d, "N": N,
-                   "blocks": (N + 63) // 64, "k_per_head": sorted(set(kph)),
-                   "merge_r": wl.r, "merge_window": list(win) if win else None, "per_gpu": "one layer instance per GPU (heads/batch shard, no collective)",
-                   "l2": "inputs larger than L2 (q,k,v,o = %.0f MB per step), no flush" % (4 * q.numel() * 2 / 1e6)},
+        "config": make_config(wl, win),
         "breakdown_ms": {"token_merge": float(seg_mean[0]), "block_scores": float(seg_mean[1]),
                          "select_blocks": float(seg_mean[2]), "sparse_attn_fwd": attn_ms,
                          "token_unmerge": float(seg_mean[4]),
                          "sparse_attn_fwd_min": float(seg[:, 3].min())},
         "effective_tflops": {"attn_kernel": attn_eff_tflops,
                              "step": eff_f / (ms_step * 1e-3) / 1e12,
+                             "note": "effective = only the selected blocks' FLOPs; `value` is the dense-equivalent "
+                                     "figure (the work dense attention would have done / step time) and is not a "
+                                     "hardware rate",
                              "frac_of_measured_burst": attn_eff_tflops / peak,
                              "frac_of_measured_sustained": attn_eff_tflops / peaks["bf16_tflops_sustained"],
                              "frac_of_nominal_2250": attn_eff_tflops / NOMINAL_BF16_TFLOPS},
-        "hbm": {"block_scores_GBps": pool_bytes / (seg_mean[1] * 1e-3) / 1e9,
-                "block_scores_frac": pool_bytes / (seg_mean[1] * 1e-3) / 1e9 / hbm},
-        "roofline": {"bound": "tensor", "kernel": "sparse_attn_fwd",
+        "roofline": {"bound": "tensor", "kernel": "sparse_attn_fwd (pair_plan_kernel + attn_pair_kernel)",
                      "achieved": attn_eff_tflops, "peak": peak, "unit": "TFLOP/s",
                      "frac": attn_eff_tflops / peak, "peak_source": "%s (burst bf16)" % peak_src,
-                     "traffic": ATTN_DRAM_TRAFFIC.get(wl.name)},
+                     "traffic": attn_dram_traffic(wl.name)},
+        "hbm_rooflines": hbm_list,
         "e2e": {"value": job_value(world, dense_f, e2e_ms), "unit": "TFLOP/s",
                 "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": int(3 * hq.numel() * 2), "d2h_bytes_per_step": int(ho.numel() * 2)},
-        "gpu_launches": launches_per_step * args.steps,
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "path": ("H2D z, metric -> merge -> projection (harness) -> scores -> select -> attention -> "
+                         "unmerge -> D2H y") if merging else "H2D q,k,v -> scores -> select -> attention -> D2H o"},
+        "gpu_launches": int(launches),
+        "gpu_launches_source": "usv_kernel_launches(): the library's own counter around the timed steps",
         "attn_entropy_ms": entropy_ms,
         "clocks": clocks,
         "context": PAPER_CONTEXT,
     }
     if merging:
         mb = (wl.B * wl.N * wl.C * 2) + (wl.B * N * wl.C * 2)
-        result["hbm"]["token_unmerge_GBps"] = mb / (seg_mean[4] * 1e-3) / 1e9
-        result["hbm"]["token_unmerge_frac"] = result["hbm"]["token_unmerge_GBps"] / hbm
+        hbm_list.append(hbm_entry("usv_token_unmerge", "unmerge_kernel", mb, float(seg_mean[4]), hbm))
+    if not args.no_merge_pass and world == 1:
+        # the HBM half of the target lives on the merge path, which the headline workload does not
+        # run: a short secondary pass on the 50 %-merge workload supplies those figures
+        extra, cfg = merge_path_rooflines(usv, device, hbm)
+        result["hbm_rooflines"] += extra
+        result["hbm_rooflines_merge_workload"] = cfg
+        assert usv.workspace_status() == 0
     return result, dict(q=q, k=k, v=v, N=N, kph=kph)
 
 
@@ -342,7 +445,9 @@ def cpu_baseline(wl, tensors, n_qb=384):
 
 
 def run_reference(args, wl):
-    """The fp64 oracle as it stands, on host cores, same metric; each step a bounded sample."""
+    """The fp64 oracle as it stands, on host cores, same metric.  The first timed step runs the
+    whole call (every query block) when that fits in about a minute and a half; every other step
+    is a bounded sample of the attention, extrapolated linearly, and says so."""
     import oracle
     q, k, v = ui.make_qkv(wl, device="cpu", layout="bhnd") if wl.merge_part is None else (None,) * 3
     if q is None:
@@ -357,23 +462,57 @@ def run_reference(args, wl):
     N, kph = wl.N_attn, wl.k_per_head()
     dense_f, _ = flops(wl, N, kph)
     n_qb = 96
-    est = []
+    est, full_steps = [], 0
+    total = picked = 0
     for i in range(args.warmup + args.steps):
         t_sel, t_attn, total, picked = oracle_sample_step(wl, q, k, v, N, kph, n_qb, i)
+        t_est = t_sel + t_attn * total / picked
+        if i == args.warmup and t_est <= 90.0 and picked < total:
+            # one whole, un-sampled step
+            t_sel, t_attn, total, _ = oracle_sample_step(wl, q, k, v, N, kph, total, i)
+            t_est = t_sel + t_attn
+            full_steps = 1
+        elif i >= args.warmup and picked >= total:
+            full_steps += 1                      # small workload: the "sample" is every query block
         if i >= args.warmup:
-            est.append(t_sel + t_attn * total / picked)
+            est.append(t_est)
     t_full = float(np.mean(est))
     val = dense_f / t_full / 1e12
-    sample = ("each step: pooling+scores+selection in full, attention on %d of %d query blocks, "
-              "extrapolated linearly to the full call" % (picked, total))
+    sample = ("pooling+scores+selection in full every step; attention: %d step(s) over all %d query blocks "
+              "(measured), %d step(s) on %d of %d query blocks extrapolated linearly to the full call"
+              % (full_steps, total, len(est) - full_steps, min(n_qb, total), total))
     return {"impl": "reference", "metric": "sparse_attn_dense_equiv_tflops", "value": val,
             "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": t_full * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "d": wl.d, "N": N},
+            "config": make_config(wl),
+            "measured_full_steps": full_steps, "extrapolated_steps": len(est) - full_steps,
+            "extrapolated": full_steps < len(est),
+            "ms_full_step_measured": est[0] * 1e3 if full_steps else None,
             "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.num_threads(),
                              "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def spawn_ranks(argv, n):
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script (one per GPU,
+    rendezvous on 127.0.0.1), pass rank 0's JSON line through, return the worst exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + argv, env=env,
+                                      stdout=subprocess.PIPE if r == 0 else subprocess.DEVNULL, text=True))
+    out, _ = procs[0].communicate()
+    rc = procs[0].returncode
+    for p_ in procs[1:]:
+        rc = max(rc, p_.wait())
+    sys.stdout.write(out)
+    return rc
 
 
 def main():
@@ -384,8 +523,15 @@ def main():
     ap.add_argument("--workload", default="wan1.3b_480p")
     ap.add_argument("--impl", default="usv", choices=["usv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-merge-pass", action="store_true",
+                    help="skip the secondary pass that times the merge-path calls for the HBM rooflines")
     ap.add_argument("--with-entropy", action="store_true",
                     help="also time usv_attn_entropy (Sec. 3.4) on the step's q, k, sel; reported beside the step")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
+                    help="process-group backend of the N > 1 path (gloo + --host-check exercise its host logic on CPU)")
+    ap.add_argument("--host-check", action="store_true",
+                    help="no GPU work: every rank contributes made-up timings to the max-over-ranks exchange and "
+                         "rank 0 prints the resulting line (tests the N > 1 plumbing on CPU)")
     ap.add_argument("--merge-window", default=None,
                     help="wt,wh,ww: keep the merge matching inside nearby partition blocks (usv arm only)")
     args = ap.parse_args()
@@ -400,13 +546,31 @@ def main():
             print(json.dumps(run_reference(args, wl)))
         return 0
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(sys.argv[1:], args.gpus)     # no launcher: be one
+
+    if args.host_check:
+        if world > 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            torch.distributed.init_process_group(args.backend, rank=rank, world_size=world)
+        ms = max_over_ranks([1.0 + rank, 10.0 - rank], world, torch.device("cpu"))
+        dense_f, _ = flops(wl, wl.N_attn, wl.k_per_head())
+        if rank == 0:
+            print(json.dumps({"host_check": True, "n_gpus": world, "ms_per_step": ms[0],
+                              "value": job_value(world, dense_f, ms[0]), "max_over_ranks": ms,
+                              "config": make_config(wl)}))
+        if world > 1:
+            torch.distributed.barrier()
+            torch.distributed.destroy_process_group()
+        return 0
+
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the CUDA library is the product and has no CPU fallback")
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.distributed.init_process_group("nccl", device_id=device)
+        torch.distributed.init_process_group(args.backend, device_id=device)
     out = run_usv(args, wl, rank, world, device)
     if rank == 0:
         result, tensors = out

@@ -62,6 +62,9 @@ const char* usv_status_string(int status);
 const char* usv_last_error(void);
 /* Compiled-in build tag, e.g. "usv-b200 sm_100a". */
 const char* usv_build_info(void);
+/* Kernels this library has launched in the calling process so far (all threads, all devices;
+ * memsets and copies are not counted). */
+unsigned long long usv_kernel_launches(void);
 
 /* ------------------------------------------------------------------------------------------
  * Coarse stage of "top-k cube selection" (Fig. 2 caption; the paper names the step and leaves

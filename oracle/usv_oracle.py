@@ -13,6 +13,13 @@ Function -> passage of the paper (equations numbered in order of appearance):
                                               neighbouring 3D blocks), the other reading of Eq. 8-9
   cube_order / select_blocks_local          : Fig. 2 caption (tokens grouped into local 3D cubes;
                                               attention in the own cube beside the top-k cubes)
+  select_blocks_long_range / attn_combine   : Fig. 2 caption, the two-branch form: local cube
+                                              attention and long-range top-k attention computed
+                                              apart, their outputs fused.  The caption does not
+                                              say how; the reading here weights each branch by
+                                              its softmax mass (parity unpinned by the paper; the
+                                              pins are the mathematics: it equals one attention
+                                              over the union of the two disjoint key sets).
 """
 import ctypes
 import os
@@ -30,7 +37,7 @@ __all__ = [
     "block_scores", "select_blocks", "dense_masked_attn", "sparse_attn", "destination_mask",
     "merge_descriptors", "merge_match", "merge_select", "merge_positions", "merge_plan",
     "merge_apply", "unmerge", "all_query_blocks", "keep_count", "key_marginal", "entropy", "allocate",
-    "cube_order", "select_blocks_local", "merge_match_local",
+    "cube_order", "select_blocks_local", "merge_match_local", "select_blocks_long_range", "attn_combine",
 ]
 
 
@@ -386,6 +393,52 @@ def select_blocks_local(scores, k_per_head):
                     a_, b_ = s[b, h, i, others[n_other - 1]], s[b, h, i, others[n_other]]
                     gap[b, h, i] = (a_ - b_) / max(abs(a_), abs(b_), 1e-30)
     return sel, gap
+
+
+def select_blocks_long_range(scores, k_per_head):
+    """Long-range branch of the two-branch form: for query block I the k_h best key blocks OTHER
+    than block I (ties -> lowest index), ascending, -1 tail.  Where fewer than k_h other blocks
+    exist all of them are kept.  Returns (sel, gap) like select_blocks_local."""
+    s = np.ascontiguousarray(scores, dtype=np.float64)
+    B, H, NBq, NBk = s.shape
+    kph = np.asarray(k_per_head, dtype=np.int64)
+    kmax = int(kph.max())
+    sel = np.full((B, H, NBq, kmax), -1, dtype=np.int32)
+    gap = np.full((B, H, NBq), np.inf)
+    for b in range(B):
+        for h in range(H):
+            k = int(kph[h])
+            for i in range(NBq):
+                others = [j for j in range(NBk) if j != i]
+                others.sort(key=lambda j: (-s[b, h, i, j], j))
+                keep = others[:k]
+                sel[b, h, i, :len(keep)] = sorted(keep)
+                if 0 < k < len(others):
+                    a_, b_ = s[b, h, i, others[k - 1]], s[b, h, i, others[k]]
+                    gap[b, h, i] = (a_ - b_) / max(abs(a_), abs(b_), 1e-30)
+    return sel, gap
+
+
+def attn_combine(o1, lse1, o2, lse2):
+    """Fusion of two attention branches over DISJOINT key sets (reading of the Fig. 2 caption):
+    each branch's output is a softmax average over its own keys and lse its log-sum-exp, so the
+    attention over both key sets together is the average of the two outputs weighted by
+    exp(lse): o = (e^lse1 o1 + e^lse2 o2) / (e^lse1 + e^lse2), lse = log(e^lse1 + e^lse2).
+    A branch without keys has lse = -inf and weight 0.  o*: [..., d], lse*: [...] -> (o, lse) fp64."""
+    o1 = np.asarray(o1, dtype=np.float64)
+    o2 = np.asarray(o2, dtype=np.float64)
+    l1 = np.asarray(lse1, dtype=np.float64)
+    l2 = np.asarray(lse2, dtype=np.float64)
+    m = np.maximum(l1, l2)
+    m_safe = np.where(np.isfinite(m), m, 0.0)
+    w1 = np.exp(l1 - m_safe)
+    w2 = np.exp(l2 - m_safe)
+    tot = w1 + w2
+    with np.errstate(invalid="ignore", divide="ignore"):
+        o = (w1[..., None] * o1 + w2[..., None] * o2) / tot[..., None]
+        lse = m_safe + np.log(tot)
+    o = np.where(tot[..., None] > 0, o, 0.0)
+    return o, lse
 
 
 def merge_match_local(mhat, grid, part, window):

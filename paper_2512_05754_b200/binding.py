@@ -45,6 +45,7 @@ def lib():
     L.usv_status_string.restype = ctypes.c_char_p
     L.usv_last_error.restype = ctypes.c_char_p
     L.usv_build_info.restype = ctypes.c_char_p
+    L.usv_kernel_launches.restype = ctypes.c_ulonglong
     for name in ("usv_block_scores_workspace", "usv_sparse_attn_workspace",
                  "usv_token_merge_workspace"):
         getattr(L, name).restype = ctypes.c_size_t
@@ -54,6 +55,11 @@ def lib():
 
 def build_info():
     return lib().usv_build_info().decode()
+
+
+def kernel_launches():
+    """Kernels the library has launched in this process so far."""
+    return int(lib().usv_kernel_launches())
 
 
 def _ptr(t):

@@ -8,6 +8,9 @@
 namespace usv {
 
 static thread_local char g_err[512] = "";
+static unsigned long long g_launches = 0;
+
+void note_launch() { __atomic_fetch_add(&g_launches, 1ull, __ATOMIC_RELAXED); }
 
 int fail(int code, const char* fmt, ...) {
     va_list ap;
@@ -43,6 +46,10 @@ extern "C" const char* usv_status_string(int status) {
 }
 
 extern "C" const char* usv_last_error(void) { return usv::g_err; }
+
+extern "C" unsigned long long usv_kernel_launches(void) {
+    return __atomic_load_n(&usv::g_launches, __ATOMIC_RELAXED);
+}
 
 extern "C" const char* usv_build_info(void) { return "usv-b200 sm_100a " __DATE__; }
 

@@ -25,8 +25,12 @@ constexpr size_t WS_HEADER = 256;
 // Validates a [B,H,N,d] view: pointer and strides 16-byte aligned, non-overlapping rows.
 int check_view(const char* name, const void* p, const usv_strides* s, int d);
 
+// Counts a kernel launch of this library (read back by usv_kernel_launches).
+void note_launch();
+
 #define USV_CHECK_LAUNCH(what)                                                              \
     do {                                                                                    \
+        usv::note_launch();                                                                 \
         cudaError_t e__ = cudaGetLastError();                                               \
         if (e__ != cudaSuccess)                                                             \
             return usv::fail(USV_ERR_CUDA, "%s: %s", (what), cudaGetErrorString(e__));      \

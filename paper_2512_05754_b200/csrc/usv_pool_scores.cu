@@ -2,7 +2,9 @@
 //
 //   pool_kernel   : one CTA per (tensor, b, h, four blocks); 16-byte loads, the next block in
 //                   flight while the current one is reduced (fp32 tree), mean over the VALID
-//                   rows of a block.
+//                   rows of a block.  At d = 128 it also writes the three bf16 planes
+//                   (mean = hi + mid + lo) that the tensor-core score kernel multiplies, so the
+//                   fp32 means are not read back for a separate split pass.
 //   scores_kernel : fp32 CUDA-core NT GEMM per (b,h), 64x64 output tile, 4x4 per thread.
 //                   Kept in fp32 (not bf16 tensor cores) because the result decides an integer
 //                   (the top-k set) that is compared with an fp64 evaluation.
@@ -16,6 +18,10 @@ struct PoolArgs {
     int N[2], NB[2];
     float* out[2];  // [B,H,NB,d]
     int H;
+    // d = 128 with the tensor-core score kernel: bf16 planes [3][B*H][NB_pad][128] per tensor
+    // (NULL: not wanted); rows NB .. NB_pad - 1 are written as zero
+    __nv_bfloat16* planes[2];
+    int NB_pad[2];
 };
 
 // D = head dim (64 or 128).  Threads: 128.  A row of D bf16 is D/8 uint4; TPR threads per row.
@@ -73,10 +79,31 @@ __global__ void __launch_bounds__(128) pool_kernel(const PoolArgs a) {
             float s = 0.f;
 #pragma unroll
             for (int g = 0; g < RPI; ++g) s += rd[g][threadIdx.x];
-            a.out[which][((int64_t)bh * NB + I) * D + threadIdx.x] = s / (float)nvalid;
+            const float mean = s / (float)nvalid;
+            a.out[which][((int64_t)bh * NB + I) * D + threadIdx.x] = mean;
+            if (a.planes[which] != nullptr) {
+                const int64_t plane = (int64_t)gridDim.y * a.NB_pad[which] * D;
+                __nv_bfloat16* dst = a.planes[which] + ((int64_t)bh * a.NB_pad[which] + I) * D + threadIdx.x;
+                float rem = mean;
+#pragma unroll
+                for (int p = 0; p < 3; ++p) {
+                    const __nv_bfloat16 hp = __float2bfloat16_rn(rem);
+                    dst[p * plane] = hp;
+                    rem -= __bfloat162float(hp);
+                }
+            }
         }
 #pragma unroll
         for (int it = 0; it < ITERS; ++it) v[it] = vn[it];
+    }
+    // the CTA that pooled the last block also clears the padding rows of the planes
+    if (I1 == NB && a.planes[which] != nullptr && threadIdx.x < D) {
+        const int64_t plane = (int64_t)gridDim.y * a.NB_pad[which] * D;
+        for (int I = NB; I < a.NB_pad[which]; ++I) {
+            __nv_bfloat16* dst = a.planes[which] + ((int64_t)bh * a.NB_pad[which] + I) * D + threadIdx.x;
+#pragma unroll
+            for (int p = 0; p < 3; ++p) dst[p * plane] = __float2bfloat16_rn(0.f);
+        }
     }
 }
 
@@ -181,16 +208,18 @@ extern "C" int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void*
     a.N[0] = Nq; a.N[1] = Nk; a.NB[0] = NBq; a.NB[1] = NBk;
     a.out[0] = qbar; a.out[1] = kbar;
     a.H = H;
+    a.planes[0] = a.planes[1] = nullptr;
+    a.NB_pad[0] = a.NB_pad[1] = 0;
+    void* tc_mem = reinterpret_cast<char*>(kbar) + align_up((size_t)B * H * NBk * d * sizeof(float), 256);
+    if (d == 128) scores_tc_planes(tc_mem, B * H, NBq, NBk, &a.planes[0], &a.planes[1], &a.NB_pad[0], &a.NB_pad[1]);
     dim3 pg(ceil_div(NBq > NBk ? NBq : NBk, POOL_SPAN), B * H, 2);
     if (d == 128) pool_kernel<128><<<pg, 128, 0, st>>>(a);
     else pool_kernel<64><<<pg, 128, 0, st>>>(a);
     USV_CHECK_LAUNCH("pool_kernel");
 
-    if (d == 128) {
-        void* mem = reinterpret_cast<char*>(kbar) + align_up((size_t)B * H * NBk * d * sizeof(float), 256);
-        return launch_scores_tc(qbar, kbar, scores, B * H, NBq, NBk, 1.0f / sqrtf((float)d), mem,
+    if (d == 128)
+        return launch_scores_tc(scores, B * H, NBq, NBk, 1.0f / sqrtf((float)d), tc_mem,
                                 static_cast<unsigned int*>(ws), st);
-    }
     dim3 sg(ceil_div(NBk, 64), ceil_div(NBq, 64), B * H);
     scores_kernel<<<sg, 256, 0, st>>>(qbar, kbar, scores, NBq, NBk, d, 1.0f / sqrtf((float)d));
     USV_CHECK_LAUNCH("scores_kernel");
@@ -265,6 +294,8 @@ extern "C" int usv_block_scores_noalloc(int B, int H, int Nq, int Nk, int d, con
     a.N[0] = Nq; a.N[1] = Nk; a.NB[0] = NBq; a.NB[1] = NBk;
     a.out[0] = qbar; a.out[1] = kbar;
     a.H = H;
+    a.planes[0] = a.planes[1] = nullptr;
+    a.NB_pad[0] = a.NB_pad[1] = 0;
     dim3 pg(ceil_div(NBq > NBk ? NBq : NBk, POOL_SPAN), B * H, 2);
     if (d == 128) pool_kernel<128><<<pg, 128, 0, st>>>(a);
     else pool_kernel<64><<<pg, 128, 0, st>>>(a);

@@ -35,42 +35,11 @@ constexpr uint32_t TA = 0, TD = NPL * 64;               // A planes at 0, 64, 12
 
 struct Args {
     int BH, NBq, NBk, NBq_pad, NBk_pad;
-    const float *qbar, *kbar;           // [BH][NB][128] fp32
     __nv_bfloat16 *a_pl, *b_pl;         // [NPL][BH][NB_pad][128]
     float* scores;                      // [BH][NBq][NBk]
     float scale;
     unsigned int* status;
 };
-
-// one warp per padded row: fp32 -> three bf16 planes (rows beyond NB are zero)
-__global__ void __launch_bounds__(256) split3_kernel(const Args m) {
-    const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    const int64_t rows_a = (int64_t)m.BH * m.NBq_pad, rows_b = (int64_t)m.BH * m.NBk_pad;
-    if (gw >= rows_a + rows_b) return;
-    const bool is_b = gw >= rows_a;
-    const int64_t rr = is_b ? gw - rows_a : gw;
-    const int pad = is_b ? m.NBk_pad : m.NBq_pad, cnt = is_b ? m.NBk : m.NBq;
-    const int bh = (int)(rr / pad), i = (int)(rr % pad);
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (i < cnt) v = *reinterpret_cast<const float4*>((is_b ? m.kbar : m.qbar) + ((int64_t)bh * cnt + i) * DM + lane * 4);
-    const float x[4] = {v.x, v.y, v.z, v.w};
-    __nv_bfloat16 pl[NPL][4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        float rem = x[e];
-#pragma unroll
-        for (int p = 0; p < NPL; ++p) {
-            pl[p][e] = __float2bfloat16_rn(rem);
-            rem -= __bfloat162float(pl[p][e]);
-        }
-    }
-    __nv_bfloat16* base = is_b ? m.b_pl : m.a_pl;
-    const int64_t plane = (is_b ? rows_b : rows_a) * DM;
-#pragma unroll
-    for (int p = 0; p < NPL; ++p)
-        *reinterpret_cast<uint2*>(base + p * plane + rr * DM + lane * 4) = *reinterpret_cast<const uint2*>(pl[p]);
-}
 
 struct Maps {
     CUtensorMap b[NPL];
@@ -267,18 +236,22 @@ size_t scores_tc_bytes(int BH, int NBq, int NBk) {
     return align_up((size_t)BH * ((size_t)pad128(NBq) + pad128(NBk)) * sc::DM * sc::NPL * sizeof(__nv_bfloat16), 256);
 }
 
-int launch_scores_tc(const float* qbar, const float* kbar, float* scores, int BH, int NBq, int NBk, float scale,
-                     void* mem, unsigned int* status, cudaStream_t st) {
+void scores_tc_planes(void* mem, int BH, int NBq, int NBk, __nv_bfloat16** a_pl, __nv_bfloat16** b_pl,
+                      int* NBq_pad, int* NBk_pad) {
+    *NBq_pad = pad128(NBq);
+    *NBk_pad = pad128(NBk);
+    *a_pl = static_cast<__nv_bfloat16*>(mem);
+    *b_pl = *a_pl + (size_t)sc::NPL * BH * *NBq_pad * sc::DM;
+}
+
+int launch_scores_tc(float* scores, int BH, int NBq, int NBk, float scale, void* mem, unsigned int* status,
+                     cudaStream_t st) {
     sc::Args m;
-    m.BH = BH; m.NBq = NBq; m.NBk = NBk; m.NBq_pad = pad128(NBq); m.NBk_pad = pad128(NBk);
-    m.qbar = qbar; m.kbar = kbar; m.scores = scores; m.scale = scale;
+    m.BH = BH; m.NBq = NBq; m.NBk = NBk;
+    m.scores = scores; m.scale = scale;
     m.status = status;
-    m.a_pl = static_cast<__nv_bfloat16*>(mem);
-    m.b_pl = m.a_pl + (size_t)sc::NPL * BH * m.NBq_pad * sc::DM;
+    scores_tc_planes(mem, BH, NBq, NBk, &m.a_pl, &m.b_pl, &m.NBq_pad, &m.NBk_pad);
     cudaError_t e;
-    const int64_t rows = (int64_t)BH * (m.NBq_pad + m.NBk_pad);
-    sc::split3_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(m);
-    USV_CHECK_LAUNCH("split3_kernel");
     sc::Maps maps;
     const int64_t brows = (int64_t)BH * m.NBk_pad;
     for (int p = 0; p < sc::NPL; ++p) {

@@ -55,3 +55,20 @@ def test_reference_arm_runs_on_rank_zero_only():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
                         "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    """`bench.py --gpus 2` run plainly (no torchrun) starts two ranks, which meet on 127.0.0.1 over
+    gloo, exchange their timings and print ONE line with n_gpus = 2 and the slowest rank's time."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--host-check",
+                        "--backend", "gloo", "--workload", "tiny"], env=env, capture_output=True, text=True,
+                       timeout=300)
+    assert r.returncode == 0, r.stderr
+    lines = [l for l in r.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2
+    assert d["max_over_ranks"] == [2.0, 10.0]          # rank 1 is slower on [0], rank 0 on [1]
+    assert d["config"]["workload"] == "tiny"
