@@ -277,6 +277,34 @@ int usv_cube_order(int T, int Hh, int W, int ct, int ch, int cw, int32_t* perm, 
                    void* stream);
 int usv_force_own_block(int B, int H, int NBq, int NBk, float* scores, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * The two-branch form of the same figure (Fig. 2 caption: local cube attention and the long-range
+ * top-k attention run apart and their outputs are fused).  The caption does not say how the
+ * outputs are fused; the reading implemented weights each branch by its softmax mass, which makes
+ * the fused output EQUAL to one attention over the union of the two branches' key sets as long as
+ * those sets are disjoint:
+ *     o = (e^lse1 o1 + e^lse2 o2) / (e^lse1 + e^lse2),    lse = log(e^lse1 + e^lse2).
+ * Recipe: local branch = usv_sparse_attn_fwd with sel[b,h,I,0] = I (k = 1); long-range branch =
+ * usv_exclude_own_block on a copy of the scores, usv_select_blocks with k - 1, usv_sparse_attn_fwd;
+ * both with lse; then usv_attn_combine.  (After token merging the branches run on the merged
+ * sequence and the fused output goes through usv_token_unmerge: "broadcast back to the full grid".)
+ *
+ * usv_exclude_own_block: scores[b,h,I,I] = -inf for I < min(NBq, NBk), in place, so that
+ * usv_select_blocks never keeps a query block's own block (as long as k < NBk).
+ *
+ * usv_attn_combine: o1, o2: branch outputs, views [B,H,N,d] (element strides, d contiguous) of
+ * bf16 (inputs_f32 = 0) or fp32 (inputs_f32 = 1, e.g. the o_f32 outputs of the branches: strides
+ * (H*N*d, N*d, d)); lse1, lse2: fp32 [B,H,N] from the branches (-inf or any value with weight 0
+ * for a branch without keys: its output is then ignored, NaN included).  o: bf16 view (written);
+ * o_f32: optional fp32 [B,H,N,d] contiguous; lse: optional fp32 [B,H,N].  A row both of whose
+ * branches are empty gets zeros and lse = -inf.
+ */
+int usv_exclude_own_block(int B, int H, int NBq, int NBk, float* scores, void* stream);
+int usv_attn_combine(int B, int H, int N, int d, const void* o1, const usv_strides* s1,
+                     const float* lse1, const void* o2, const usv_strides* s2, const float* lse2,
+                     int inputs_f32, void* o, const usv_strides* so, float* o_f32, float* lse,
+                     void* stream);
+
 #ifdef __cplusplus
 }
 #endif

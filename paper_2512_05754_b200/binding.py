@@ -368,3 +368,43 @@ def force_own_block(scores):
     B, H, NBq, NBk = scores.shape
     _check(lib().usv_force_own_block(B, H, NBq, NBk, _ptr(scores), _stream(scores.device)), "usv_force_own_block")
     return scores
+
+
+def exclude_own_block(scores):
+    """In place: scores[b,h,I,I] = -inf, so that select_blocks never keeps a query block's own block
+    (the long-range branch of the two-branch form)."""
+    if scores.dtype != torch.float32 or not scores.is_contiguous() or not scores.is_cuda or scores.dim() != 4:
+        raise ValueError("scores must be a contiguous CUDA fp32 [B,H,NBq,NBk] tensor")
+    B, H, NBq, NBk = scores.shape
+    _check(lib().usv_exclude_own_block(B, H, NBq, NBk, _ptr(scores), _stream(scores.device)), "usv_exclude_own_block")
+    return scores
+
+
+def attn_combine(o1, lse1, o2, lse2, out=None, return_f32=False, return_lse=False):
+    """Fuses two attention branches over disjoint key sets by their softmax mass.  o1, o2: [B,H,N,d]
+    views, both bf16 or both fp32; lse1, lse2: fp32 [B,H,N].  Returns o (bf16) [, o_f32] [, lse]."""
+    if o1.dtype != o2.dtype or o1.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("o1 and o2 must both be bf16 or both be fp32")
+    for t in (o1, o2):
+        if t.dim() != 4 or not t.is_cuda or t.stride(3) != 1:
+            raise ValueError("branch outputs must be CUDA [B,H,N,d] views with a contiguous last axis")
+    B, H, N, d = o1.shape
+    for l in (lse1, lse2):
+        if l.dtype != torch.float32 or not l.is_contiguous() or tuple(l.shape) != (B, H, N):
+            raise ValueError("lse must be a contiguous fp32 [B,H,N] tensor")
+    s1 = _Strides(o1.stride(0), o1.stride(1), o1.stride(2))
+    s2 = _Strides(o2.stride(0), o2.stride(1), o2.stride(2))
+    if out is None:
+        out = torch.empty((B, H, N, d), dtype=torch.bfloat16, device=o1.device)
+    so = _view(out, "o")
+    o32 = torch.empty((B, H, N, d), dtype=torch.float32, device=o1.device) if return_f32 else None
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=o1.device) if return_lse else None
+    _check(lib().usv_attn_combine(B, H, N, d, _ptr(o1), ctypes.byref(s1), _ptr(lse1), _ptr(o2), ctypes.byref(s2),
+                                  _ptr(lse2), 1 if o1.dtype == torch.float32 else 0, _ptr(out), ctypes.byref(so),
+                                  _ptr(o32), _ptr(lse), _stream(o1.device)), "usv_attn_combine")
+    res = (out,)
+    if return_f32:
+        res += (o32,)
+    if return_lse:
+        res += (lse,)
+    return res if len(res) > 1 else out

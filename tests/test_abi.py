@@ -78,6 +78,18 @@ def test_argument_validation_happens_on_the_host(L):
     assert L.usv_cube_order(0, 3, 4, 4, 4, 4, p, None, None) == 1
     assert L.usv_cube_order(2, 3, 4, 4, 4, 4, None, None, None) == 1
     assert L.usv_force_own_block(1, 2, 4, 4, None, None) == 1
+    # two-branch fusion: null scores; unsupported head width; null log-sum-exp; bad input-type flag
+    assert L.usv_exclude_own_block(1, 2, 4, 4, None, None) == 1
+    assert L.usv_attn_combine(1, 2, 128, 96, p, ctypes.byref(s), p, p, ctypes.byref(s), p, 0, p, ctypes.byref(s), None,
+                              None, None) == 2
+    assert L.usv_attn_combine(1, 2, 128, 128, p, ctypes.byref(s), None, p, ctypes.byref(s), p, 0, p, ctypes.byref(s),
+                              None, None, None) == 1
+    assert L.usv_attn_combine(1, 2, 128, 128, p, ctypes.byref(s), p, p, ctypes.byref(s), p, 7, p, ctypes.byref(s),
+                              None, None, None) == 1
+    # status helpers: null workspace
+    assert L.usv_workspace_init(None, None) == 1
+    assert L.usv_workspace_status(None, None) == 1
+    assert L.usv_selftest_wait_timeout(p, 0, None) == 1
 
 
 def test_workspace_sizes(L):
