@@ -142,12 +142,12 @@ def job_value(world, flops_per_rank, ms_per_step):
     return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
 
 
-def make_config(wl, merge_window=None):
+def make_config(wl, merge_window=None, fused_unmerge=False):
     """The workload description both arms print (identical keys and values)."""
     N = wl.N_attn
     return {"workload": wl.name, "B": wl.B, "H": wl.H, "d": wl.d, "N": N, "blocks": (N + 63) // 64,
             "k_per_head": sorted(set(wl.k_per_head())), "merge_r": wl.r,
-            "merge_window": list(merge_window) if merge_window else None,
+            "merge_window": list(merge_window) if merge_window else None, "fused_unmerge": bool(fused_unmerge),
             "per_gpu": "one layer instance per GPU (heads/batch shard, no collective)",
             "l2": ("inputs larger than L2 (q,k,v,o = %.0f MB per step), no flush" if 4 * wl.B * wl.H * N * wl.d * 2 > 126e6
                    else "q,k,v,o = %.1f MB per step: fits in L2, not flushed (sanity workload)")
@@ -239,20 +239,28 @@ def run_usv(args, wl, rank, world, device):
         o = torch.empty_like(q)
 
     marks = []
+    fused = merging and args.fused_unmerge and wl.d == 128
+    y_full = torch.empty((wl.B, wl.N, wl.C), dtype=torch.bfloat16, device=device) if fused else None
 
     def step(record=False):
         e = [ev() for _ in range(6)] if record else None
         if record: e[0].record()
+        umap = None
         if merging:
-            usv.token_merge(inp["z"], inp["metric"], wl.grid, wl.merge_part, wl.r, window=win)
+            _, pl = usv.token_merge(inp["z"], inp["metric"], wl.grid, wl.merge_part, wl.r, window=win)
+            if fused:
+                umap = usv.unmerge_map(pl.pos, N)      # inverse of the plan's pos, part of building the plan
         if record: e[1].record()
         s = usv.block_scores(q, k, N, N)
         if record: e[2].record()
         sel = usv.select_blocks(s, kph)
         if record: e[3].record()
-        usv.sparse_attn_fwd(q, k, v, sel, kph, N=N, out=o)
+        if fused:
+            usv.sparse_attn_fwd_unmerge(q, k, v, sel, kph, umap, wl.N, N=N, out=y_full)
+        else:
+            usv.sparse_attn_fwd(q, k, v, sel, kph, N=N, out=o)
         if record: e[4].record()
-        if merging:
+        if merging and not fused:
             usv.token_unmerge(o.permute(0, 2, 1, 3).reshape(wl.B, N, wl.C), plan.pos)
         if record:
             e[5].record()
@@ -372,7 +380,7 @@ def run_usv(args, wl, rank, world, device):
         "vs_baseline": None,
         "dtype": "bf16",
         "data": "synthetic",
-        "config": make_config(wl, win),
+        "config": make_config(wl, win, fused),
         "breakdown_ms": {"token_merge": float(seg_mean[0]), "block_scores": float(seg_mean[1]),
                          "select_blocks": float(seg_mean[2]), "sparse_attn_fwd": attn_ms,
                          "token_unmerge": float(seg_mean[4]),
@@ -527,6 +535,9 @@ def main():
                     help="skip the secondary pass that times the merge-path calls for the HBM rooflines")
     ap.add_argument("--with-entropy", action="store_true",
                     help="also time usv_attn_entropy (Sec. 3.4) on the step's q, k, sel; reported beside the step")
+    ap.add_argument("--fused-unmerge", action="store_true",
+                    help="merging workloads: unmerge inside the attention epilogue (usv_sparse_attn_fwd_unmerge) "
+                         "instead of a separate usv_token_unmerge call")
     ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
                     help="process-group backend of the N > 1 path (gloo + --host-check exercise its host logic on CPU)")
     ap.add_argument("--host-check", action="store_true",

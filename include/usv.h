@@ -156,6 +156,34 @@ int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_str
                         int kmax, void* o, const usv_strides* so, float* o_f32, float* lse,
                         float scale, int impl, void* ws, size_t ws_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Attention with the unmerge of Eq. 15 folded into its epilogue (Sec. 3.3: after attention every
+ * merged row is sent back to all the original positions it stands for).  Same computation as
+ * usv_sparse_attn_fwd on the merged sequence of N tokens, but every output row is stored straight
+ * to the original tokens that read it back, y[b, n, h*d ... h*d+d) for every n with pos[b,n] = row,
+ * so that no separate usv_token_unmerge pass (a read of the merged output and a launch) is needed.
+ *
+ * usv_unmerge_map builds the inverse of pos once per merge plan (any pos works, e.g. a cube
+ * permutation): unmerge_off int32 [B, Nm+1] (offsets), unmerge_idx int32 [B, N] (original tokens
+ * grouped by merged row).  ws: usv_unmerge_map_workspace(B, Nm) bytes.
+ *
+ * usv_sparse_attn_fwd_unmerge: arguments as usv_sparse_attn_fwd (tcgen05 kernel only: d = 128);
+ * N = merged length, N_full = original length, y: bf16 [B, N_full, H*d] contiguous (written: every
+ * token whose pos lies in [0, N)).  o is still required: it receives the (normally zero) query
+ * blocks that are recomputed exactly before they are copied to y, and is otherwise left
+ * undefined.  o_f32 / lse, if given, are written in the merged order as usual.
+ */
+size_t usv_unmerge_map_workspace(int B, int Nm);
+int usv_unmerge_map(int B, int N, int Nm, const int32_t* pos, int32_t* unmerge_off, int32_t* unmerge_idx,
+                    void* ws, size_t ws_bytes, void* stream);
+int usv_sparse_attn_fwd_unmerge(int B, int H, int N, int d, const void* q, const usv_strides* sq,
+                                const void* k, const usv_strides* sk, const void* v,
+                                const usv_strides* sv, const int32_t* sel, const int32_t* k_per_head,
+                                int kmax, void* o, const usv_strides* so, float* o_f32, float* lse,
+                                float scale, void* ws, size_t ws_bytes, int N_full,
+                                const int32_t* unmerge_off, const int32_t* unmerge_idx, void* y,
+                                void* stream);
+
 /* After usv_sparse_attn_fwd with impl 0: how many query blocks the tcgen05 kernel handed to the
  * exact kernel because their softmax sums left the safe exponent range (normally 0).
  * Synchronises `stream`.  ws is the workspace that call used. */

@@ -47,7 +47,7 @@ def lib():
     L.usv_build_info.restype = ctypes.c_char_p
     L.usv_kernel_launches.restype = ctypes.c_ulonglong
     for name in ("usv_block_scores_workspace", "usv_sparse_attn_workspace",
-                 "usv_token_merge_workspace"):
+                 "usv_token_merge_workspace", "usv_unmerge_map_workspace"):
         getattr(L, name).restype = ctypes.c_size_t
     _lib = L
     return L
@@ -402,6 +402,55 @@ def attn_combine(o1, lse1, o2, lse2, out=None, return_f32=False, return_lse=Fals
     _check(lib().usv_attn_combine(B, H, N, d, _ptr(o1), ctypes.byref(s1), _ptr(lse1), _ptr(o2), ctypes.byref(s2),
                                   _ptr(lse2), 1 if o1.dtype == torch.float32 else 0, _ptr(out), ctypes.byref(so),
                                   _ptr(o32), _ptr(lse), _stream(o1.device)), "usv_attn_combine")
+    res = (out,)
+    if return_f32:
+        res += (o32,)
+    if return_lse:
+        res += (lse,)
+    return res if len(res) > 1 else out
+
+
+def unmerge_map(pos, Nm):
+    """Inverse of pos [B,N] (int32): (unmerge_off int32 [B,Nm+1], unmerge_idx int32 [B,N]), the
+    original tokens grouped by the merged row they read back.  Built once per merge plan."""
+    if pos.dtype != torch.int32 or not pos.is_contiguous() or not pos.is_cuda or pos.dim() != 2:
+        raise ValueError("pos must be a contiguous CUDA int32 [B,N] tensor")
+    B, N = pos.shape
+    off = torch.empty((B, Nm + 1), dtype=torch.int32, device=pos.device)
+    idx = torch.empty((B, N), dtype=torch.int32, device=pos.device)
+    L = lib()
+    ws = _workspace(pos.device, L.usv_unmerge_map_workspace(B, int(Nm)))
+    _check(L.usv_unmerge_map(B, N, int(Nm), _ptr(pos), _ptr(off), _ptr(idx), _ptr(ws), ctypes.c_size_t(ws.numel()),
+                             _stream(pos.device)), "usv_unmerge_map")
+    return off, idx
+
+
+def sparse_attn_fwd_unmerge(q, k, v, sel, k_per_head, umap, N_full, N=None, scale=0.0, out=None,
+                            return_f32=False, return_lse=False):
+    """sparse_attn_fwd on the merged sequence with the unmerge folded into its epilogue: returns
+    y bf16 [B,N_full,H*d] (every original token holds the output row of its merged row) and, if
+    asked for, the fp32 output / log-sum-exp in merged order.  umap = unmerge_map(plan.pos, N)."""
+    sq, sk, sv = _view(q, "q"), _view(k, "k"), _view(v, "v")
+    B, H, n, d = q.shape
+    N = n if N is None else int(N)
+    off, idx = umap
+    if tuple(off.shape) != (B, N + 1) or tuple(idx.shape) != (B, int(N_full)):
+        raise ValueError("unmerge map does not fit (B, N, N_full)")
+    kmax = sel.shape[3]
+    karr, _ = _k_array(k_per_head, H)
+    if out is None:
+        out = torch.empty((B, int(N_full), H * d), dtype=torch.bfloat16, device=q.device)
+    scratch = torch.empty((B, n, H, d), dtype=q.dtype, device=q.device).permute(0, 2, 1, 3)
+    so = _view(scratch, "o")
+    o32 = torch.empty((B, H, N, d), dtype=torch.float32, device=q.device) if return_f32 else None
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if return_lse else None
+    L = lib()
+    ws = _workspace(q.device, L.usv_sparse_attn_workspace(B, H, N, d, kmax))
+    _check(L.usv_sparse_attn_fwd_unmerge(B, H, N, d, _ptr(q), ctypes.byref(sq), _ptr(k), ctypes.byref(sk),
+                                         _ptr(v), ctypes.byref(sv), _ptr(sel), karr, kmax, _ptr(scratch),
+                                         ctypes.byref(so), _ptr(o32), _ptr(lse), ctypes.c_float(scale), _ptr(ws),
+                                         ctypes.c_size_t(ws.numel()), int(N_full), _ptr(off), _ptr(idx), _ptr(out),
+                                         _stream(q.device)), "usv_sparse_attn_fwd_unmerge")
     res = (out,)
     if return_f32:
         res += (o32,)

@@ -23,6 +23,13 @@ struct AttnArgs {
     const int* lists;
     int64_t list_batch;
     int64_t list_off[USV_MAX_HEADS];
+    // Fused unmerge (NULL / 0 when off): the tcgen05 kernel stores every output row to all the
+    // original tokens that read it back, y[b, n, h*d ...] for n in unmerge_idx[b, off[row] .. off[row+1]),
+    // instead of to o.  y: bf16 [B, N_full, H*d] contiguous.
+    const int32_t* unmerge_off;   // [B, N+1]
+    const int32_t* unmerge_idx;   // [B, N_full]
+    __nv_bfloat16* y;
+    int N_full;
     const int* work_list;   // list mode of the exact kernel (NULL = one CTA per query block)
     const int* work_count;
     int B, H, N, NB, kmax;
@@ -34,6 +41,8 @@ struct AttnArgs {
 int launch_attn_mma(const AttnArgs& a, int d, cudaStream_t st);
 bool attn_pair_supported(const AttnArgs& a, int d);
 int launch_attn_pair(const AttnArgs& a, int d, cudaStream_t st);
+// fused unmerge: copies the query blocks the exact kernel recomputed (into o) to their original tokens in y
+int launch_scatter_fallbacks(const AttnArgs& a, int d, cudaStream_t st);
 // ints one pair's list occupies for a head that keeps k of NB key blocks (header + entries)
 __host__ __device__ inline int64_t list_stride(int k, int NB) { return 1 + (int64_t)(2 * (int64_t)k < NB ? 2 * k : NB); }
 size_t pair_plan_bytes(int B, int H, int NB, const int32_t* k_per_head);

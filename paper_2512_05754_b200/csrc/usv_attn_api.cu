@@ -15,13 +15,22 @@ extern "C" size_t usv_sparse_attn_workspace(int B, int H, int N, int d, int kmax
     return usv::WS_HEADER + usv::align_up((size_t)B * H * NB * sizeof(int), 256) + usv::pair_plan_bytes(B, H, NB, kk);
 }
 
-extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,
-                                   const void* k, const usv_strides* sk, const void* v,
-                                   const usv_strides* sv, const int32_t* sel,
-                                   const int32_t* k_per_head, int kmax, void* o,
-                                   const usv_strides* so, float* o_f32, float* lse, float scale,
-                                   int impl, void* ws, size_t ws_bytes, void* stream) {
+static int sparse_attn_impl(int B, int H, int N, int d, const void* q, const usv_strides* sq,
+                            const void* k, const usv_strides* sk, const void* v,
+                            const usv_strides* sv, const int32_t* sel,
+                            const int32_t* k_per_head, int kmax, void* o,
+                            const usv_strides* so, float* o_f32, float* lse, float scale,
+                            int impl, void* ws, size_t ws_bytes, void* stream, int N_full,
+                            const int32_t* unmerge_off, const int32_t* unmerge_idx, void* y) {
     using namespace usv;
+    if (y != nullptr) {
+        if (unmerge_off == nullptr || unmerge_idx == nullptr)
+            return fail(USV_ERR_INVALID_ARG, "sparse_attn_unmerge: null unmerge map");
+        if (N_full < N) return fail(USV_ERR_INVALID_ARG, "sparse_attn_unmerge: N_full=%d < N=%d", N_full, N);
+        if (d != 128 || impl != 0)
+            return fail(USV_ERR_UNSUPPORTED, "sparse_attn_unmerge: the fused unmerge needs d = 128 and impl 0");
+        if (!aligned16(y)) return fail(USV_ERR_UNSUPPORTED, "sparse_attn_unmerge: y not 16-byte aligned");
+    }
     if (B <= 0 || H <= 0 || N <= 0) return fail(USV_ERR_INVALID_ARG, "sparse_attn: B,H,N must be positive");
     if (d != 64 && d != 128) return fail(USV_ERR_UNSUPPORTED, "sparse_attn: d=%d (need 64 or 128)", d);
     if (H > USV_MAX_HEADS) return fail(USV_ERR_UNSUPPORTED, "sparse_attn: H > %d", USV_MAX_HEADS);
@@ -70,6 +79,10 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
     a.list_batch = 0;
     a.work_list = nullptr;
     a.work_count = nullptr;
+    a.unmerge_off = unmerge_off;
+    a.unmerge_idx = unmerge_idx;
+    a.y = static_cast<__nv_bfloat16*>(y);
+    a.N_full = N_full;
     a.B = B; a.H = H; a.N = N; a.NB = NB; a.kmax = kmax;
     const float sc = scale == 0.f ? 1.0f / sqrtf((float)d) : scale;
     a.scale_log2 = sc * 1.4426950408889634f;
@@ -85,7 +98,32 @@ extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, co
         // exact recomputation of the (normally zero) query blocks the fast kernel reported
         a.work_list = a.fallback_list;
         a.work_count = a.fallback_count;
-        return launch_attn_mma(a, d, st);
+        rc2 = launch_attn_mma(a, d, st);
+        if (rc2 != USV_OK || y == nullptr) return rc2;
+        return launch_scatter_fallbacks(a, d, st);
     }
+    if (y != nullptr) return fail(USV_ERR_UNSUPPORTED, "sparse_attn_unmerge: sequence too long for the tcgen05 kernel");
     return launch_attn_mma(a, d, st);
+}
+
+extern "C" int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,
+                                   const void* k, const usv_strides* sk, const void* v,
+                                   const usv_strides* sv, const int32_t* sel,
+                                   const int32_t* k_per_head, int kmax, void* o,
+                                   const usv_strides* so, float* o_f32, float* lse, float scale,
+                                   int impl, void* ws, size_t ws_bytes, void* stream) {
+    return sparse_attn_impl(B, H, N, d, q, sq, k, sk, v, sv, sel, k_per_head, kmax, o, so, o_f32, lse, scale, impl, ws,
+                            ws_bytes, stream, 0, nullptr, nullptr, nullptr);
+}
+
+extern "C" int usv_sparse_attn_fwd_unmerge(int B, int H, int N, int d, const void* q, const usv_strides* sq,
+                                           const void* k, const usv_strides* sk, const void* v,
+                                           const usv_strides* sv, const int32_t* sel,
+                                           const int32_t* k_per_head, int kmax, void* o,
+                                           const usv_strides* so, float* o_f32, float* lse, float scale,
+                                           void* ws, size_t ws_bytes, int N_full, const int32_t* unmerge_off,
+                                           const int32_t* unmerge_idx, void* y, void* stream) {
+    if (y == nullptr) return usv::fail(USV_ERR_INVALID_ARG, "sparse_attn_unmerge: null y");
+    return sparse_attn_impl(B, H, N, d, q, sq, k, sk, v, sv, sel, k_per_head, kmax, o, so, o_f32, lse, scale, 0, ws,
+                            ws_bytes, stream, N_full, unmerge_off, unmerge_idx, y);
 }

@@ -214,6 +214,12 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                         const int grow = Ir * USV_BLOCK + (rr & 63);
                         if (Ir >= 0 && grow < N) {
                             *reinterpret_cast<uint4*>(O + (int64_t)grow * a.so.sn + cc * 8) = make_uint4(0, 0, 0, 0);
+                            if (a.y != nullptr) {
+                                const int u1 = a.unmerge_off[(int64_t)b * (N + 1) + grow + 1];
+                                for (int u = a.unmerge_off[(int64_t)b * (N + 1) + grow]; u < u1; ++u)
+                                    *reinterpret_cast<uint4*>(a.y + ((int64_t)b * a.N_full + a.unmerge_idx[(int64_t)b * a.N_full + u]) *
+                                                                        ((int64_t)a.H * D) + h * D + cc * 8) = make_uint4(0, 0, 0, 0);
+                            }
                             const int64_t grow_bh = ((int64_t)b * a.H + h) * N + grow;
                             if (a.o_f32 != nullptr) {
                                 float4* o32 = reinterpret_cast<float4*>(a.o_f32 + grow_bh * D + cc * 8);
@@ -519,6 +525,12 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
             // accumulator and the ring slot go back as soon as the last quarter has been read.
             float* o32 = (a.o_f32 != nullptr && live) ? a.o_f32 + (((int64_t)ib * a.H + ih) * N + row) * D : nullptr;
             __nv_bfloat16* O = a.o + ib * a.so.sb + ih * a.so.sh + (int64_t)row * a.so.sn;
+            // fused unmerge: the row goes to every original token that reads it back
+            int u0 = 0, u1 = 0;
+            if (a.y != nullptr && live) {
+                u0 = a.unmerge_off[(int64_t)ib * (N + 1) + row];
+                u1 = a.unmerge_off[(int64_t)ib * (N + 1) + row + 1];
+            }
 #pragma unroll 1
             for (int qd = 0; qd < 4; ++qd) {
                 uint32_t r0[32];
@@ -540,13 +552,24 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
                                         __uint_as_float(r0[4 * j + 2]) * inv, __uint_as_float(r0[4 * j + 3]) * inv);
                 }
                 if (live) {
+                    uint4 pk[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
-                        *reinterpret_cast<uint4*>(O + qd * 32 + 8 * i) =
-                            make_uint4(pack_bf16x2(__uint_as_float(r0[8 * i]) * inv, __uint_as_float(r0[8 * i + 1]) * inv),
-                                       pack_bf16x2(__uint_as_float(r0[8 * i + 2]) * inv, __uint_as_float(r0[8 * i + 3]) * inv),
-                                       pack_bf16x2(__uint_as_float(r0[8 * i + 4]) * inv, __uint_as_float(r0[8 * i + 5]) * inv),
-                                       pack_bf16x2(__uint_as_float(r0[8 * i + 6]) * inv, __uint_as_float(r0[8 * i + 7]) * inv));
+                        pk[i] = make_uint4(pack_bf16x2(__uint_as_float(r0[8 * i]) * inv, __uint_as_float(r0[8 * i + 1]) * inv),
+                                           pack_bf16x2(__uint_as_float(r0[8 * i + 2]) * inv, __uint_as_float(r0[8 * i + 3]) * inv),
+                                           pack_bf16x2(__uint_as_float(r0[8 * i + 4]) * inv, __uint_as_float(r0[8 * i + 5]) * inv),
+                                           pack_bf16x2(__uint_as_float(r0[8 * i + 6]) * inv, __uint_as_float(r0[8 * i + 7]) * inv));
+                    if (a.y == nullptr) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(O + qd * 32 + 8 * i) = pk[i];
+                    } else {
+                        for (int u = u0; u < u1; ++u) {
+                            const int tok = a.unmerge_idx[(int64_t)ib * a.N_full + u];
+                            __nv_bfloat16* Y = a.y + ((int64_t)ib * a.N_full + tok) * ((int64_t)a.H * D) + ih * D + qd * 32;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(Y + 8 * i) = pk[i];
+                        }
+                    }
                 }
             }
         }
@@ -674,7 +697,36 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     }
 }
 
+// Fused unmerge: query blocks the exact kernel recomputed sit in o; copy them to their tokens in y.
+__global__ void __launch_bounds__(128) scatter_fallback_kernel(const AttnArgs a) {
+    const int count = *a.fallback_count;
+    const int NB = a.NB, N = a.N;
+    for (int w = blockIdx.x; w < count; w += gridDim.x) {
+        const int id = a.fallback_list[w];
+        const int I = id % NB, bh_ord = id / NB;
+        const int b = bh_ord / a.H, h = a.head_order[bh_ord % a.H];
+        for (int idx = threadIdx.x; idx < USV_BLOCK * (D / 8); idx += 128) {
+            const int rr = idx / (D / 8), cc = idx % (D / 8);
+            const int row = I * USV_BLOCK + rr;
+            if (row >= N) continue;
+            const uint4 val = *reinterpret_cast<const uint4*>(a.o + b * a.so.sb + h * a.so.sh + (int64_t)row * a.so.sn + cc * 8);
+            const int u0 = a.unmerge_off[(int64_t)b * (N + 1) + row], u1 = a.unmerge_off[(int64_t)b * (N + 1) + row + 1];
+            for (int u = u0; u < u1; ++u) {
+                const int tok = a.unmerge_idx[(int64_t)b * a.N_full + u];
+                *reinterpret_cast<uint4*>(a.y + ((int64_t)b * a.N_full + tok) * ((int64_t)a.H * D) + h * D + cc * 8) = val;
+            }
+        }
+    }
+}
+
 }  // namespace pr
+
+int launch_scatter_fallbacks(const AttnArgs& a, int d, cudaStream_t st) {
+    (void)d;
+    pr::scatter_fallback_kernel<<<64, 128, 0, st>>>(a);
+    USV_CHECK_LAUNCH("scatter_fallback_kernel");
+    return USV_OK;
+}
 
 bool attn_pair_supported(const AttnArgs& a, int d) {
     return d == pr::D && a.NB <= pr::MAX_NB && a.work_counter != nullptr;

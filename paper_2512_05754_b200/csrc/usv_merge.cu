@@ -576,6 +576,27 @@ __global__ void __launch_bounds__(256) unmerge_kernel(int N, int Nm, int C,
     for (int c = lane; c < nvec; c += 32) dst[c] = __ldg(src + c);
 }
 
+// ---------------------------------------------------------------------------- unmerge map
+// Inverse of pos: for every merged row the original tokens that read it back (counting sort by
+// merged row; the order inside a row is irrelevant, every token of a row receives the same values).
+__global__ void __launch_bounds__(256) inv_count_kernel(int N, int Nm, const int32_t* __restrict__ pos,
+                                                        int32_t* __restrict__ cnt) {
+    const int b = blockIdx.y;
+    const int n = blockIdx.x * 256 + threadIdx.x;
+    if (n >= N) return;
+    const int m = pos[(int64_t)b * N + n];
+    if (m >= 0 && m < Nm) atomicAdd(&cnt[(int64_t)b * Nm + m], 1);
+}
+
+__global__ void __launch_bounds__(256) inv_fill_kernel(int N, int Nm, const int32_t* __restrict__ pos,
+                                                       int32_t* __restrict__ cursor, int32_t* __restrict__ inv_idx) {
+    const int b = blockIdx.y;
+    const int n = blockIdx.x * 256 + threadIdx.x;
+    if (n >= N) return;
+    const int m = pos[(int64_t)b * N + n];
+    if (m >= 0 && m < Nm) inv_idx[(int64_t)b * N + atomicAdd(&cursor[(int64_t)b * Nm + m], 1)] = n;
+}
+
 // ---------------------------------------------------------------------------- host side
 struct MergeWs {
     size_t mhat, src_idx, jstar_s, u_s, row_src, cnt, off, cursor, csr, status, tsel, split, total;
@@ -729,6 +750,35 @@ extern "C" int usv_token_unmerge(int B, int N, int Nm, int C, const void* y_merg
         N, Nm, C, static_cast<const __nv_bfloat16*>(y_merged), pos,
         static_cast<__nv_bfloat16*>(y), rows);
     USV_CHECK_LAUNCH("unmerge_kernel");
+    return USV_OK;
+}
+
+extern "C" size_t usv_unmerge_map_workspace(int B, int Nm) {
+    if (B <= 0 || Nm <= 0) return 0;
+    return usv::WS_HEADER + 2 * usv::align_up((size_t)B * Nm * sizeof(int32_t), 256);
+}
+
+extern "C" int usv_unmerge_map(int B, int N, int Nm, const int32_t* pos, int32_t* inv_off, int32_t* inv_idx,
+                               void* ws, size_t ws_bytes, void* stream) {
+    using namespace usv;
+    if (B <= 0 || N <= 0 || Nm <= 0 || Nm > N) return fail(USV_ERR_INVALID_ARG, "unmerge_map: need B,N,Nm > 0 and Nm <= N");
+    if (pos == nullptr || inv_off == nullptr || inv_idx == nullptr || ws == nullptr)
+        return fail(USV_ERR_INVALID_ARG, "unmerge_map: null pointer");
+    if (B > 65535) return fail(USV_ERR_UNSUPPORTED, "unmerge_map: B > 65535");
+    if (ws_bytes < usv_unmerge_map_workspace(B, Nm))
+        return fail(USV_ERR_WORKSPACE, "unmerge_map: workspace %zu < %zu", ws_bytes, usv_unmerge_map_workspace(B, Nm));
+    int32_t* cnt = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + WS_HEADER);
+    int32_t* cursor = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + WS_HEADER + align_up((size_t)B * Nm * 4, 256));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(cnt, 0, (size_t)B * Nm * 4, s);
+    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "unmerge_map: memset: %s", cudaGetErrorString(e));
+    dim3 tg(ceil_div(N, 256), B);
+    inv_count_kernel<<<tg, 256, 0, s>>>(N, Nm, pos, cnt);
+    USV_CHECK_LAUNCH("inv_count_kernel");
+    csr_scan_kernel<<<dim3(ceil_div(Nm, 1024), B), 1024, 0, s>>>(Nm, cnt, inv_off, cursor);
+    USV_CHECK_LAUNCH("csr_scan_kernel");
+    inv_fill_kernel<<<tg, 256, 0, s>>>(N, Nm, pos, cursor, inv_idx);
+    USV_CHECK_LAUNCH("inv_fill_kernel");
     return USV_OK;
 }
 
