@@ -11,9 +11,10 @@
 //
 // The row is mapped to order-preserving 32-bit keys in shared memory.  Four 8-bit radix passes
 // (most significant digit first) find the key T of the k-th largest element and the number of
-// elements strictly above it.  A final ordered pass emits, in ascending block index, every
-// index whose key is above T plus the first (k - above) indices whose key equals T, which is
-// exactly "k largest, ties to the lowest index".
+// elements strictly above it.  The output pass gives every thread a contiguous stretch of the
+// row: it counts what it keeps (every key above T, and the first (k - above) keys equal to T,
+// which is exactly "k largest, ties to the lowest index"), one block-wide scan places it, and it
+// writes its indices in ascending order.  Rows that keep everything skip the search.
 #include "usv_common.cuh"
 
 namespace usv {
@@ -49,11 +50,11 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* __rest
                                                              int32_t* __restrict__ sel, int H,
                                                              int NBq, int NBk, int kmax,
                                                              const SelHeads heads) {
-    __shared__ uint32_t keys[SEL_MAX_NB];
+    extern __shared__ uint32_t keys[];   // NBk order-preserving keys
     __shared__ int hist[256];
     __shared__ int scratch[9];
     __shared__ uint32_t s_prefix;
-    __shared__ int s_remaining;
+    __shared__ int s_remaining, s_eq_total;
 
     const int row = blockIdx.x;  // (b*H + h)*NBq + I
     const int h = (row / NBq) % H;
@@ -61,6 +62,11 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* __rest
     const float* src = scores + (int64_t)row * NBk;
     int32_t* out = sel + (int64_t)row * kmax;
 
+    if (k >= NBk) {   // keep everything: no search
+        for (int j = threadIdx.x; j < NBk; j += SEL_THREADS) out[j] = j;
+        for (int t = NBk + threadIdx.x; t < kmax; t += SEL_THREADS) out[t] = -1;
+        return;
+    }
     for (int j = threadIdx.x; j < NBk; j += SEL_THREADS) keys[j] = float_key(src[j]);
     if (threadIdx.x == 0) {
         s_prefix = 0;
@@ -97,6 +103,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* __rest
                 if (before < remaining && remaining <= before + local[t]) {
                     s_prefix = prefix | ((uint32_t)(255 - (lane * 8 + t)) << shift);
                     s_remaining = remaining - before;
+                    s_eq_total = local[t];   // after the last pass: how many keys equal T
                 }
                 before += local[t];
             }
@@ -105,20 +112,38 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* __rest
     }
     const uint32_t T = s_prefix;
     const int need_eq = s_remaining;  // how many elements equal to T are kept (lowest indices)
+    const bool all_eq = need_eq == s_eq_total;   // no tie straddles the cut (the usual case)
 
-    int base_out = 0, base_eq = 0;
-    for (int j0 = 0; j0 < NBk; j0 += SEL_THREADS) {
-        const int j = j0 + threadIdx.x;
-        const uint32_t key = j < NBk ? keys[j] : 0u;
-        const int is_gt = (j < NBk && key > T) ? 1 : 0;
-        const int is_eq = (j < NBk && key == T) ? 1 : 0;
-        int tot_eq, tot_out;
-        const int eq_rank = base_eq + block_excl_scan(is_eq, scratch, &tot_eq);
-        const int take = is_gt | (is_eq && eq_rank < need_eq);
-        const int p = base_out + block_excl_scan(take, scratch, &tot_out);
-        if (take) out[p] = j;
-        base_eq += tot_eq;
-        base_out += tot_out;
+    // Ordered output.  Thread t owns the contiguous indices [t L, t L + L): it counts what it keeps,
+    // one block-wide scan gives its first output slot, and it writes its indices in order.
+    const int L = (NBk + SEL_THREADS - 1) / SEL_THREADS;
+    const int j0 = threadIdx.x * L, j1 = min(j0 + L, NBk);
+    int eq_base = 0;
+    if (!all_eq) {   // ties across the cut: the lowest indices among the equal keys win
+        int ne = 0;
+        for (int j = j0; j < j1; ++j) ne += keys[j] == T ? 1 : 0;
+        int tot;
+        eq_base = block_excl_scan(ne, scratch, &tot);
+    }
+    int cnt = 0;
+    {
+        int eq_seen = eq_base;
+        for (int j = j0; j < j1; ++j) {
+            const uint32_t key = keys[j];
+            if (key > T) ++cnt;
+            else if (key == T) { if (all_eq || eq_seen < need_eq) ++cnt; ++eq_seen; }
+        }
+    }
+    int tot_out;
+    int p = block_excl_scan(cnt, scratch, &tot_out);
+    {
+        int eq_seen = eq_base;
+        for (int j = j0; j < j1; ++j) {
+            const uint32_t key = keys[j];
+            bool take = key > T;
+            if (key == T) { take = all_eq || eq_seen < need_eq; ++eq_seen; }
+            if (take) out[p++] = j;
+        }
     }
     for (int t = k + threadIdx.x; t < kmax; t += SEL_THREADS) out[t] = -1;
 }
@@ -126,7 +151,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* __rest
 // One warp per row; lane l holds the scores of indices i * 32 + l, i < KPL (every load of the
 // row is one contiguous 128-byte line per warp).
 template <int KPL>
-__global__ void __launch_bounds__(256) select_warp_kernel(const float* __restrict__ scores,
+__global__ void __launch_bounds__(256, 2) select_warp_kernel(const float* __restrict__ scores,
                                                           int32_t* __restrict__ sel, int H, int NBq,
                                                           int NBk, int kmax, const SelHeads heads,
                                                           int64_t rows) {
@@ -138,15 +163,31 @@ __global__ void __launch_bounds__(256) select_warp_kernel(const float* __restric
     const int k = heads.k[h];
     const float* src = scores + row * NBk;
     int32_t* out = sel + row * kmax;
+    if (k >= NBk) {   // keep everything: no search (uniform over the warp)
+        for (int j = lane; j < NBk; j += 32) out[j] = j;
+        for (int t = NBk + lane; t < kmax; t += 32) out[t] = -1;
+        return;
+    }
     uint32_t key[KPL];
 #pragma unroll
     for (int i = 0; i < KPL; ++i) key[i] = (i * 32 + lane < NBk) ? float_key(__ldg(src + i * 32 + lane)) : 0u;   // 0 < any real key
     // Largest T with count(key >= T) >= k, one bit at a time.  As soon as a candidate leaves
     // exactly k keys at or above it, those k are the answer and no tie can straddle the cut.
-    uint32_t T = 0;
+    // The bits above the highest one in which two real keys differ are common to all of them and
+    // to T: the search starts below them.
+    uint32_t kor = 0u, kand = 0xffffffffu;
+#pragma unroll
+    for (int i = 0; i < KPL; ++i)
+        if (i * 32 + lane < NBk) { kor |= key[i]; kand &= key[i]; }
+    kor = __reduce_or_sync(0xffffffffu, kor);
+    kand = __reduce_and_sync(0xffffffffu, kand);
+    const uint32_t diff = kor ^ kand;
+    const int top = diff ? 31 - __clz(diff) : -1;               // highest differing bit (-1: all keys equal)
+    uint32_t T = top >= 31 ? 0u : (kand & ~((2u << (top < 0 ? 0 : top)) - 1u));
+    if (top < 0) T = kand;
     bool exact = false;
 #pragma unroll 1
-    for (int bit = 31; bit >= 0; --bit) {
+    for (int bit = top; bit >= 0; --bit) {
         const uint32_t cand = T | (1u << bit);
         int c = 0;
 #pragma unroll
@@ -213,7 +254,7 @@ extern "C" int usv_select_blocks(int B, int H, int NBq, int NBk, const float* sc
     else if (NBk <= 1024) USV_SEL_WARP(32);
     else if (NBk <= 1536) USV_SEL_WARP(48);
     else if (NBk <= 2048) USV_SEL_WARP(64);
-    else select_kernel<<<(unsigned)rows, SEL_THREADS, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads);
+    else select_kernel<<<(unsigned)rows, SEL_THREADS, (size_t)NBk * sizeof(uint32_t), st>>>(scores, sel, H, NBq, NBk, kmax, heads);
 #undef USV_SEL_WARP
     USV_CHECK_LAUNCH("select_kernel");
     return USV_OK;

@@ -167,13 +167,21 @@ def test_select_kernel_exact_on_tied_scores(usv):
     g = torch.Generator().manual_seed(11)
     # rows up to 2048 scores take the warp-per-row kernel, longer ones the CTA-per-row kernel
     for NBk, ks in ((16, [1, 16, 5]), (300, [7, 150, 299]), (1393, [70, 349, 1393]), (2048, [1, 2048, 777]),
-                    (2500, [3, 1250, 2500])):
+                    (2500, [3, 1250, 2500]), (3023, [152, 1, 3022]), (4096, [205, 4096, 2048]), (8192, [1, 410, 8191])):
         s = torch.randint(-3, 4, (2, 3, 9, NBk), generator=g).float()
         s[0, 0, 0] = 0.0
         s[1, 2, 3] = -0.0
         sel = usv.select_blocks(s.to(_dev()), ks).cpu().numpy()
         ref, _ = oracle.select_blocks(s.double().numpy(), ks)
         assert np.array_equal(sel, ref)
+        # the same rows with all scores of a row equal but for a few (the search's common-prefix
+        # start, and a cut that falls inside one long run of equal keys)
+        s2 = torch.full_like(s, 1.5)
+        s2[..., ::7] = 2.5
+        s2[0, 1, 2] = -3.0
+        sel2 = usv.select_blocks(s2.to(_dev()), ks).cpu().numpy()
+        ref2, _ = oracle.select_blocks(s2.double().numpy(), ks)
+        assert np.array_equal(sel2, ref2)
 
 
 def test_unselected_blocks_are_never_read(usv):
