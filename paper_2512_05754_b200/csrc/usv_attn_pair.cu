@@ -22,26 +22,28 @@
 // logits.  Rows whose sum leaves [2^-100, 2^100] are reported in a list and recomputed by the
 // exact online-softmax kernel, so the result never depends on that assumption.
 //
-// One persistent CTA per SM, 19 warps, draws items from a global counter (heads with long lists
+// One persistent CTA per SM, 24 warps, draws items from a global counter (heads with long lists
 // first).  Every role runs straight on from one item into the next, so that the tensor pipe
 // only drains at the end of the kernel:
 //   warps 0-15   four softmax warpgroups sharing the 128 rows (thread r of every group <-> TMEM
 //                lane r <-> query row r).  Group g works on the tiles of running parity g >> 1
-//                and there on key block g & 1 of the tile (64 logit columns).  The same threads
-//                write an item's output: each reads its row's 32 columns of O (group g: columns
-//                32 g ...) out of TMEM, hands the accumulator back and stores from registers.
-//                A group may take one tile of the next item before it turns to the output of
-//                the last one, so that the pipe finds new weights while the last P.V finishes.
-//   warp 16      scout + K producer: draws the next item, copies its key-block list into a ring
+//                and there on key block g & 1 of the tile (64 logit columns).
+//   warps 16-19  output: thread e <-> query row e reads the finished O row out of TMEM a quarter at
+//                a time, hands the accumulator back and stores from registers (to o, or, with the
+//                unmerge folded in, to every original token that reads the row back), while the
+//                softmax groups are already in the next item.
+//   warp 20      scout + K producer: draws the next item, copies its key-block list into a ring
 //                slot in shared memory and publishes it, fetches Q and the K tiles (TMA).
-//   warp 17      MMA issuer and TMEM owner.
-//   warp 18      V producer (TMA).
+//   warp 21      P.V issuer and TMEM owner.
+//   warp 22      V producer (TMA).
+//   warp 23      S issuer.
+// The CTA is launched with 80 registers per thread and the roles re-divide them at their start
+// (setmaxnreg): the softmax loop needs more than the launch allows for 768 threads, the others less.
 //
 // TMEM holds O and THREE S buffers; running tile g uses buffer g mod 3.  The weights P are
 // written back, as bf16 pairs, into the columns their logits came from, so a buffer goes
-// S(g) -> P(g) -> S(g + 3) without a hand-back: P.V(g) is issued before S(g + 3), and the tensor
-// pipe runs its MMAs in issue order.  Every barrier has one set of waiters that sees each of its
-// phases (SFULL/PFULL are indexed by g mod 6, the per-item barriers by item mod 4: a waiter that
+// S(g) -> P(g) -> S(g + 3); S(g + 3) is issued once P.V(g) is complete.  Every barrier has
+// waiters that see each of its phases (SFULL/PFULL are indexed by g mod 6, the per-item barriers by item mod 4: a waiter that
 // skipped a phase could not tell it from the one two before).  All waits are bounded; a wait
 // that gives up sets the device status word and every role leaves its loop.
 #include "usv_attn.cuh"
@@ -91,8 +93,8 @@ constexpr uint32_t TO = 0, TS = 128;
 static_assert(TS + SBUF * 128 <= TMEM_COLS, "TMEM budget");
 
 constexpr int NSOFT = NWG * 128;   // softmax threads
-constexpr int NTHREADS = NSOFT + 128 + 128;   // + output warpgroup + service warpgroup (three warps used)
-constexpr int W_EPI = NSOFT / 32, W_TMA = W_EPI + 4, W_MMA = W_EPI + 5, W_TMA_V = W_EPI + 6;
+constexpr int NTHREADS = NSOFT + 128 + 128;   // + output warpgroup + service warpgroup
+constexpr int W_EPI = NSOFT / 32, W_TMA = W_EPI + 4, W_MMA = W_EPI + 5, W_TMA_V = W_EPI + 6, W_MMA_S = W_EPI + 7;
 // Registers per thread after the roles part ways (setmaxnreg, whole warpgroups).  A CTA can only
 // redistribute what it was launched with: 24 warps x 80 registers = 1920 per lane, and
 // 16 x 96 + 4 x 56 + 4 x 40 = 1920.  (A request beyond the pool would wait forever.)
@@ -350,143 +352,82 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
             if (!ok) break;
         }
     } else if (warp == W_MMA) {
-        // ===== MMA issuer (whole warp in the loop, one elected lane issues); TMEM owner =========
+        // ===== P.V issuer (whole warp in the loop, one elected lane issues); TMEM owner ==========
+        // Two warps feed the tensor pipe, this one the O += P.V tiles and W_MMA_S the S = Q.K^T tiles:
+        // while one of them waits on a barrier or does its bookkeeping, the MMAs of the other keep
+        // the pipe busy.  MMAs of different threads are ordered only through barriers: S(g) reuses the
+        // TMEM buffer of P(g - 3) and is issued once P.V(g - 3) is COMPLETE (the V stage barrier
+        // of that tile says so to the V producer and to the S issuer alike).
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REG_SERVICE));
-        // The tensor pipe takes MMAs from a short queue: the issuing thread can be about two
-        // MMAs ahead of it and no more, so every stretch of ~100 cycles it spends on anything
-        // else idles the pipe.  The loop is therefore shaped around the MMA stream: one step =
-        // P.V(g) followed by S(g + 3), sixteen MMAs back to back, and the barrier tests for the
-        // next step (non-blocking) are taken between MMAs of this one, in the shadow of the queue.
-        constexpr uint32_t IDESC_S = instr_desc(128, KT, 0, 0);    // Q (K-major) x K (K-major)
         constexpr uint32_t IDESC_O = instr_desc(128, D, 0, 1);     // P (TMEM) x V (MN-major)
+        const uint64_t vdesc0 = smem_desc(base + SM_V, 16384, 1024);
+        int g = 0;                               // running tile
+        int p_v = 0, p_buf = 0, p_b6 = 0;        // g % VSTAGES, g % SBUF, g % (2 SBUF)
+        uint32_t p_vph = 0, p_ph6 = 0;           // (g / VSTAGES) & 1, (g / (2 SBUF)) & 1
+        bool ok = true;
+        for (int n = 0; ok; ++n) {
+            if (!mbar_wait(bar(B_IFULL + n % NSLOT), (n / NSLOT) & 1, s_abort, a.status, 0x10000)) break;
+            const int T = hdr_of(n)[I_T];
+            if (T < 0) break;
+            for (int t = 0; t < T; ++t, ++g) {
+                if (!mbar_wait(bar(B_VFULL + p_v), p_vph, s_abort, a.status, 0x20)) { ok = false; break; }
+                if (!mbar_wait(bar(B_PFULL + p_b6), p_ph6, s_abort, a.status, 0x40)) { ok = false; break; }
+                // the first P.V of an item overwrites O: the item before must have been read out
+                if (t == 0 && n > 0 && !mbar_wait(bar(B_OFREE), (n - 1) & 1, s_abort, a.status, 0x2000)) { ok = false; break; }
+                fence_after();
+                const uint64_t vdesc = vdesc0 + ((p_v * TILE_BYTES) >> 4);
+                const uint32_t pb = tmem + TS + p_buf * 128;   // P: 32 columns at the head of each 64-column half
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < KT / 16; ++ks)
+                        umma_ts(tmem + TO, pb + (ks >> 2) * 64 + (ks & 3) * 8, vdesc + ((ks * 2048) >> 4), IDESC_O,
+                                (t > 0 || ks > 0));
+                    umma_commit(bar(B_VEMPTY + p_v));      // V stage free; S buffer p_buf free for S(g + 3)
+                    if (t == T - 1) umma_commit(bar(B_OFULL));
+                }
+                __syncwarp();
+                if (++p_v == VSTAGES) { p_v = 0; p_vph ^= 1; }
+                if (++p_buf == SBUF) p_buf = 0;
+                if (++p_b6 == 2 * SBUF) { p_b6 = 0; p_ph6 ^= 1; }
+            }
+        }
+    } else if (warp == W_MMA_S) {
+        // ===== S issuer ===========================================================================
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REG_SERVICE));
+        static_assert(VSTAGES == SBUF, "the V stage barrier of tile g doubles as the hand-back of S buffer g % SBUF");
+        constexpr uint32_t IDESC_S = instr_desc(128, KT, 0, 0);    // Q (K-major) x K (K-major)
         const uint64_t qdesc = smem_desc(base + SM_Q, 16, 1024);        // + byte offset >> 4
         const uint64_t kdesc0 = smem_desc(base + SM_K, 16, 1024);
-        const uint64_t vdesc0 = smem_desc(base + SM_V, 16384, 1024);
-        // Two cursors over the running sequence of tiles.  The S cursor (item sn, tile st of Ts,
-        // running index gs) runs up to SBUF tiles ahead of the P.V cursor (item n, tile t of T,
-        // running index gt) and crosses into the next item on its own, so that the pipe sees no
-        // seam between items.  S(g) goes into buffer g % SBUF; its previous tenant P(g - SBUF) is
-        // read by P.V(g - SBUF), issued before it (the tensor pipe runs its MMAs in issue order).
-        int sn = -1, st = 0, Ts = 0, gs = 0;
-        int s_k = 0, s_buf = 0, s_b6 = 0;      // gs % KSTAGES, gs % SBUF, gs % (2 SBUF)
-        uint32_t s_kph = 0;                    // (gs / KSTAGES) & 1
-        int n = 0, t = 0, T = 0, gt = 0;
-        int p_v = 0, p_buf = 0, p_b6 = 0;      // gt % VSTAGES, gt % SBUF, gt % (2 SBUF)
-        uint32_t p_vph = 0, p_ph6 = 0;         // (gt / VSTAGES) & 1, (gt / (2 SBUF)) & 1
-        bool s_done = false;              // the S cursor has met the end marker
-        unsigned long long tring = 0;     // tile counts of the last four items the S cursor entered, 16 bits each
+        int g = 0;
+        int s_k = 0, s_buf = 0, s_b6 = 0;      // g % KSTAGES, g % SBUF, g % (2 SBUF)
+        uint32_t s_kph = 0, s_bph = 1;         // (g / KSTAGES) & 1; parity of the hand-back of buffer s_buf: ((g / SBUF) & 1) ^ 1
         bool ok = true;
-        // Can S(gs) be issued?  1 yes, 0 not now (or never: end marker), -1 a bounded wait gave up.
-        // `must`: block until it can (P.V(gt) needs S(gt)).
-        auto s_ready = [&](bool must) -> int {
-            if (st == Ts) {
-                const int m = sn + 1;
-                if (!mbar_test(bar(B_IFULL + m % NSLOT), (m / NSLOT) & 1)) {
-                    if (!must) return 0;
-                    if (!mbar_wait(bar(B_IFULL + m % NSLOT), (m / NSLOT) & 1, s_abort, a.status, 0x10000)) return -1;
-                }
-                const int Tm = hdr_of(m)[I_T];
-                if (Tm < 0) { s_done = true; return 0; }
-                sn = m; st = 0; Ts = Tm;
-                tring = (tring << 16) | (unsigned)Tm;
-            }
-            if (st == 0 && !mbar_test(bar(B_QFULL), sn & 1)) {
-                if (!must) return 0;
-                if (!mbar_wait(bar(B_QFULL), sn & 1, s_abort, a.status, 0x4)) return -1;
-            }
-            if (!mbar_test(bar(B_KFULL + s_k), s_kph)) {
-                if (!must) return 0;
-                if (!mbar_wait(bar(B_KFULL + s_k), s_kph, s_abort, a.status, 0x8)) return -1;
-            }
-            return 1;
-        };
-        // MMAs k0 .. k1 - 1 of S(gs): the Q buffer, K stage s_k -> S buffer s_buf
-        auto issue_s = [&](int k0, int k1) {
-            const uint64_t kdesc = kdesc0 + ((s_k * TILE_BYTES) >> 4);
-            const uint32_t d_s = tmem + TS + s_buf * 128;
-            if (elect_one()) {
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    if (ks < k0 || ks >= k1) continue;
-                    const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
-                    umma_ss(d_s, qdesc + off, kdesc + off, IDESC_S, ks > 0);
-                }
-            }
-            __syncwarp();
-        };
-        // S(gs) is issued: completion signals, cursor on to the next tile
-        auto finish_s = [&]() {
-            if (elect_one()) {
-                umma_commit(bar(B_SFULL + s_b6));
-                umma_commit(bar(B_KEMPTY + s_k));              // its K stage may be refilled
-                if (st == Ts - 1) umma_commit(bar(B_QFREE));   // and, after an item's last tile, the Q buffer
-            }
-            __syncwarp();
-            ++st; ++gs;
-            if (++s_k == KSTAGES) { s_k = 0; s_kph ^= 1; }
-            if (++s_buf == SBUF) s_buf = 0;
-            if (++s_b6 == 2 * SBUF) s_b6 = 0;
-        };
-        bool v_rdy = false, p_rdy = false;   // V(gt) / P(gt) seen complete by an earlier test
-        for (;;) {
-            // S tiles the cursor is behind with (the first tiles of the kernel, or a K tile that was
-            // late): all of them before this thread blocks on anything else
-            while (!s_done && gs < gt + SBUF) {
-                const int sr = s_ready(gs <= gt);
-                if (sr < 0) ok = false;
-                if (sr <= 0) break;
+        for (int n = 0; ok; ++n) {
+            if (!mbar_wait(bar(B_IFULL + n % NSLOT), (n / NSLOT) & 1, s_abort, a.status, 0x10000)) break;
+            const int T = hdr_of(n)[I_T];
+            if (T < 0) break;
+            if (!mbar_wait(bar(B_QFULL), n & 1, s_abort, a.status, 0x4)) break;
+            for (int t = 0; t < T; ++t, ++g) {
+                if (!mbar_wait(bar(B_KFULL + s_k), s_kph, s_abort, a.status, 0x8)) { ok = false; break; }
+                // buffer s_buf held P(g - 3): P.V(g - 3) must be complete
+                if (g >= SBUF && !mbar_wait(bar(B_VEMPTY + s_buf), s_bph, s_abort, a.status, 0x100)) { ok = false; break; }
                 fence_after();
-                issue_s(0, D / 16);
-                finish_s();
-            }
-            if (!ok) break;
-            if (t == 0) {
-                if (sn < n) break;   // end marker: there is no item n
-                T = (int)((tring >> (16 * (sn - n))) & 0xffffu);
-            }
-            if (!v_rdy && !mbar_wait(bar(B_VFULL + p_v), p_vph, s_abort, a.status, 0x20)) break;
-            if (!p_rdy && !mbar_wait(bar(B_PFULL + p_b6), p_ph6, s_abort, a.status, 0x40)) break;
-            // the first P.V of an item overwrites O: the item before must have been read out
-            if (t == 0 && n > 0 && !mbar_wait(bar(B_OFREE), (n - 1) & 1, s_abort, a.status, 0x2000)) break;
-            fence_after();
-            const uint64_t vdesc = vdesc0 + ((p_v * TILE_BYTES) >> 4);
-            const uint32_t pb = tmem + TS + p_buf * 128;   // P: 32 columns at the head of each 64-column half
-            if (elect_one()) {
+                const uint64_t kdesc = kdesc0 + ((s_k * TILE_BYTES) >> 4);
+                const uint32_t d_s = tmem + TS + s_buf * 128;
+                if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_ts(tmem + TO, pb + (ks & 3) * 8, vdesc + ((ks * 2048) >> 4), IDESC_O, (t > 0 || ks > 0));
-            }
-            __syncwarp();
-            // S(gt + SBUF) follows this P.V if its inputs are there (tested while the pipe works)
-            int sr = 0;
-            if (!s_done && gs <= gt + SBUF) {
-                sr = s_ready(false);
-                if (sr < 0) break;
-            }
-            if (elect_one()) {
-#pragma unroll
-                for (int ks = 4; ks < KT / 16; ++ks)
-                    umma_ts(tmem + TO, pb + 64 + (ks & 3) * 8, vdesc + ((ks * 2048) >> 4), IDESC_O, 1u);
-                umma_commit(bar(B_VEMPTY + p_v));
-                if (t == T - 1) umma_commit(bar(B_OFULL));
-            }
-            __syncwarp();
-            ++gt;
-            if (++t == T) { t = 0; ++n; }
-            if (++p_v == VSTAGES) { p_v = 0; p_vph ^= 1; }
-            if (++p_buf == SBUF) p_buf = 0;
-            if (++p_b6 == 2 * SBUF) { p_b6 = 0; p_ph6 ^= 1; }
-            if (sr > 0) {
-                fence_after();
-                issue_s(0, 3);
-                v_rdy = mbar_test(bar(B_VFULL + p_v), p_vph);
-                issue_s(3, 6);
-                p_rdy = mbar_test(bar(B_PFULL + p_b6), p_ph6);
-                issue_s(6, D / 16);
-                finish_s();
-            } else {
-                v_rdy = mbar_test(bar(B_VFULL + p_v), p_vph);
-                p_rdy = mbar_test(bar(B_PFULL + p_b6), p_ph6);
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
+                        umma_ss(d_s, qdesc + off, kdesc + off, IDESC_S, ks > 0);
+                    }
+                    umma_commit(bar(B_SFULL + s_b6));
+                    umma_commit(bar(B_KEMPTY + s_k));             // its K stage may be refilled
+                    if (t == T - 1) umma_commit(bar(B_QFREE));    // and, after an item's last tile, the Q buffer
+                }
+                __syncwarp();
+                if (++s_k == KSTAGES) { s_k = 0; s_kph ^= 1; }
+                if (++s_buf == SBUF) { s_buf = 0; s_bph ^= 1; }
+                if (++s_b6 == 2 * SBUF) s_b6 = 0;
             }
         }
     } else if (warp >= W_EPI && warp < W_TMA) {
@@ -676,9 +617,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
             if (lane == 0) mbar_arrive(bar(B_SUMS + slot_n));
             g += T;
         }
-    } else {
-        // fourth warp of the service warpgroup: no role, but the register hand-over is per warpgroup
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REG_SERVICE));
     }
 
     // ---- teardown
