@@ -26,14 +26,20 @@ struct MatchTcArgs {
     Part p;
     int B, N, nA, nA_pad, nB_pad;
     const int32_t* src_idx;          // [nA] source tokens, ascending
-    __nv_bfloat16 *a_hi, *a_lo;      // [B][nA_pad][128]
-    __nv_bfloat16 *b_hi, *b_lo;      // [B][nB_pad][128]
+    uint16_t* a_h;                   // fp16 bits [B][nA_pad][128]
+    uint16_t* b_h;                   // fp16 bits [B][nB_pad][128]
+    float* cand_v;                   // [B][nA][2][4] largest approximate cosines per source and tile parity, descending
+    int* cand_i;                     // [B][nA][2][4] their destination ordinals
+    int* exact_list;                 // sources (b * nA + rank) that need the fp32 scan of all destinations
+    int* exact_count;
+    unsigned long long* exact_best;  // one slot per list entry: (key of the best cosine << 32) | ~destination
+    float* floor_v;                  // [B][nA_pad] lower bound on each source's approximate row maximum
     int32_t* jstar_s;                // [B][nA] best destination TOKEN per source rank
     float* u_s;                      // [B][nA] its cosine
     unsigned int* status;            // device status word for bounded waits (may be NULL)
 };
 
-// bytes of the hi/lo planes for a sequence of N tokens (any partition: sources + destinations = N)
+// bytes of the matcher's scratch for a sequence of N tokens (any partition: sources + destinations = N)
 size_t match_tc_bytes(int B, int N);
 // mhat: fp32 unit descriptors [B,N,128]; mem: match_tc_bytes(B, N) bytes, 256-byte aligned.
 int launch_match_tc(const float* mhat, const Part& p, int B, int N, int nA, const int32_t* src_idx,

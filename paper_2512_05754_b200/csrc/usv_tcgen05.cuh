@@ -71,6 +71,29 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// The same bounded wait, polling without ever suspending the thread (test_wait): for waits on the
+// critical path of a short producer/consumer chain, where the wake-up time of a suspended thread
+// would be a large part of every round trip.
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               unsigned int* status, unsigned int code,
+                                               unsigned long long limit_ns = WAIT_LIMIT_NS) {
+#pragma unroll 1
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_test(bar, parity)) return true;
+    const unsigned long long t0 = gtime();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 1024; ++i)
+            if (mbar_test(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (gtime() - t0 > limit_ns) {
+            *abort_flag = 1;
+            if (status) atomicOr(status, code);
+            return false;
+        }
+    }
+}
+
 // True in exactly one lane of a converged warp.  Single-thread instructions (TMA, MMA, commit)
 // are issued under it from warp-uniform code, so that their operands stay in uniform registers.
 __device__ __forceinline__ bool elect_one() {
@@ -136,6 +159,12 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
 __host__ __device__ constexpr uint32_t instr_desc(int m, int n, int a_major, int b_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_major << 15) | ((uint32_t)b_major << 16) |
            (((uint32_t)n >> 3) << 17) | (((uint32_t)m >> 4) << 24);
+}
+
+// The same for fp16 x fp16 -> fp32 (both operands of one MMA must have the same type).
+__host__ __device__ constexpr uint32_t instr_desc_f16(int m, int n, int a_major, int b_major) {
+    return (1u << 4) | ((uint32_t)a_major << 15) | ((uint32_t)b_major << 16) | (((uint32_t)n >> 3) << 17) |
+           (((uint32_t)m >> 4) << 24);
 }
 
 #define USV_R16(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), \

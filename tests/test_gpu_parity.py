@@ -260,6 +260,34 @@ def test_merge_many_sources_into_one_destination(usv):
     assert bf16_ulp_distance(bits(xm), ref).max() <= 1
 
 
+def test_matching_with_crowded_windows_dm128(usv):
+    """dm = 128 (tensor-core matcher: one fp16 product, the four best approximate cosines kept per
+    source, fp32 re-check).  Descriptors drawn from a handful of prototypes plus tiny noise put
+    dozens of destinations within the error window of every row maximum, and exact duplicates tie
+    exactly: every such source takes the fp32 scan of all destinations.  Its choice must be
+    admissible (inside the near-tie band of the oracle's maximum; bit-identical rows after the
+    bf16 rounding of the metric tie in exact arithmetic) and everything downstream must follow it."""
+    grid, part = (4, 12, 16), (1, 1, 2)                    # 768 tokens, 384 destinations
+    N = 768
+    g = torch.Generator().manual_seed(77)
+    proto = torch.randn(5, 2, 128, generator=g)
+    which = torch.randint(0, 5, (N,), generator=g)
+    metric = proto[which] + 1e-4 * torch.randn(N, 2, 128, generator=g)
+    metric[100:140] = proto[1]                             # exact duplicates, sources and destinations alike
+    metric = metric.unsqueeze(0).to(torch.bfloat16)
+    x = _rand_bf16((1, N, 64), 78)
+    for r in (0, 200, 384):
+        xm, plan = usv.token_merge(x.to(_dev()), metric.to(_dev()), grid, part, r, debug=True)
+        torch.cuda.synchronize()
+        assert usv.workspace_status() == 0
+        pg = dict(dst_of=plan.dst_of.cpu().numpy(), pos=plan.pos.cpu().numpy(),
+                  u=plan.u.cpu().numpy(), jstar=plan.jstar.cpu().numpy())
+        stats = check_merge_plan(pg, metric, grid, part, r)
+        print("crowded r=%d: %s" % (r, stats))
+        ref = oracle.round_to_bf16(oracle.merge_apply(x, pg["dst_of"], pg["pos"], N - r))
+        assert bf16_ulp_distance(bits(xm), ref).max() <= 1
+
+
 # ---------------------------------------------------------------- argument validation on device
 
 def test_errors_leave_outputs_untouched(usv):
