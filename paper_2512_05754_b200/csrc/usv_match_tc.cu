@@ -99,6 +99,13 @@ struct Maps {
     CUtensorMap b_h;
 };
 
+// maximum of three fp32 values given as bit patterns (one instruction on this architecture)
+__device__ __forceinline__ float max3(uint32_t a, uint32_t b, uint32_t c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(__uint_as_float(a)), "f"(__uint_as_float(b)), "f"(__uint_as_float(c)));
+    return d;
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -229,26 +236,30 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
             fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(B_DFREE + eg));
-            if (nvalid < 128) {
-#pragma unroll
-                for (int j = 0; j < 128; ++j)
-                    if (j >= nvalid) sr[j] = 0xff800000u;   // -inf: a destination that does not exist
-            }
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
-                // The chunk's maximum first, on four independent chains (a running compare over
-                // all 32 would be one long dependent chain); only a chunk that reaches into the window
-                // of the running maximum is gone through element by element, in ascending order (the
-                // maximum only grows, so a destination below the window can never matter).
-                float c0 = __uint_as_float(sr[ch * 32]), c1 = __uint_as_float(sr[ch * 32 + 1]),
-                      c2 = __uint_as_float(sr[ch * 32 + 2]), c3 = __uint_as_float(sr[ch * 32 + 3]);
+                if (nvalid < (ch + 1) * 32) {   // only the chunks of the last tile that reach past the end (uniform)
 #pragma unroll
-                for (int j = 4; j < 32; j += 4) {
-                    c0 = fmaxf(c0, __uint_as_float(sr[ch * 32 + j]));
-                    c1 = fmaxf(c1, __uint_as_float(sr[ch * 32 + j + 1]));
-                    c2 = fmaxf(c2, __uint_as_float(sr[ch * 32 + j + 2]));
-                    c3 = fmaxf(c3, __uint_as_float(sr[ch * 32 + j + 3]));
+                    for (int j = 0; j < 32; ++j)
+                        if (ch * 32 + j >= nvalid) sr[ch * 32 + j] = 0xff800000u;   // -inf: a destination that does not exist
                 }
+                // The chunk's maximum first (three-input maxima on four independent chains); only a
+                // chunk that reaches into the window of the running maximum is gone through element by
+                // element, in ascending order (the maximum only grows, so a destination below the
+                // window can never matter).
+                float c0 = max3(sr[ch * 32], sr[ch * 32 + 1], sr[ch * 32 + 2]);
+                float c1 = max3(sr[ch * 32 + 3], sr[ch * 32 + 4], sr[ch * 32 + 5]);
+                float c2 = max3(sr[ch * 32 + 6], sr[ch * 32 + 7], sr[ch * 32 + 8]);
+                float c3 = max3(sr[ch * 32 + 9], sr[ch * 32 + 10], sr[ch * 32 + 11]);
+#pragma unroll
+                for (int j = 12; j < 28; j += 8) {
+                    c0 = max3(__float_as_uint(c0), sr[ch * 32 + j], sr[ch * 32 + j + 1]);
+                    c1 = max3(__float_as_uint(c1), sr[ch * 32 + j + 2], sr[ch * 32 + j + 3]);
+                    c2 = max3(__float_as_uint(c2), sr[ch * 32 + j + 4], sr[ch * 32 + j + 5]);
+                    c3 = max3(__float_as_uint(c3), sr[ch * 32 + j + 6], sr[ch * 32 + j + 7]);
+                }
+                c0 = max3(__float_as_uint(c0), sr[ch * 32 + 28], sr[ch * 32 + 29]);
+                c1 = max3(__float_as_uint(c1), sr[ch * 32 + 30], sr[ch * 32 + 31]);
                 const float cm = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
                 if (cm >= fmaxf(vmax, floor_v) - 2.0f * EPS && cm > vlast) {
                     // rare: the chunk goes through shared memory so that the insertion is ONE rolled
