@@ -16,6 +16,7 @@ namespace plan {
 constexpr int ROUNDS = 6;      // upper limit; the matching stops as soon as a round finds nothing new
 constexpr int CH = 128;        // query blocks per chunk
 constexpr int THREADS = 4 * CH;
+constexpr int OVP = CH + 8;     // row pitch of the overlap matrix (uint16): rows start 4 banks apart
 
 // One CTA per chunk of CH consecutive query blocks of one (batch, head).
 //   1. bitmaps of the chunk's selection rows (shared memory)
@@ -37,8 +38,8 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
     const int NP = (NB + 1) >> 1;
     const int nwords = (NB + 31) >> 5;
     const int pitch = nwords | 1;                       // odd row pitch: rows start in different banks
-    uint16_t* ov = reinterpret_cast<uint16_t*>(smem_u);            // [CH][CH], rows 16-byte aligned
-    uint32_t* bm = smem_u + CH * CH / 2;                           // [CH][pitch]
+    uint16_t* ov = reinterpret_cast<uint16_t*>(smem_u);            // [CH][OVP], rows 16-byte aligned
+    uint32_t* bm = smem_u + CH * OVP / 2;                          // [CH][pitch]
     const int bh = blockIdx.y;
     const int b = bh / a.H, h = bh % a.H;
     const int kh = a.k_per_head[h];
@@ -68,16 +69,16 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
     __syncthreads();
     const int32_t* sel = a.sel + ((int64_t)bh * NB + I0) * a.kmax;
     const int total = nI * kh;
-    for (int i0 = threadIdx.x; i0 < total; i0 += 4 * THREADS) {
-        int J[4], R[4];
+    for (int i0 = threadIdx.x; i0 < total; i0 += 16 * THREADS) {
+        int J[16], R[16];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {          // four independent loads in flight
+        for (int u = 0; u < 16; ++u) {         // sixteen independent loads in flight
             const int i = i0 + u * THREADS;
             R[u] = i < total ? i / kh : -1;
             J[u] = i < total ? sel[(int64_t)R[u] * a.kmax + (i - R[u] * kh)] : -1;
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < 16; ++u)
             if (J[u] >= 0 && J[u] < NB) atomicOr(&bm[R[u] * pitch + (J[u] >> 5)], 1u << (J[u] & 31));
     }
     if (threadIdx.x < CH) partner[threadIdx.x] = -1;
@@ -85,20 +86,18 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
         const int first = threadIdx.x * 32;
         freebits[threadIdx.x] = first >= nI ? 0u : (nI - first >= 32 ? 0xffffffffu : (1u << (nI - first)) - 1u);
     }
-    for (int i = threadIdx.x; i < CH * CH / 2; i += THREADS) smem_u[i] = 0u;   // overlaps of blocks past the end: 0
+    for (int i = threadIdx.x; i < CH * OVP / 2; i += THREADS) smem_u[i] = 0u;   // overlaps of blocks past the end: 0
     __syncthreads();
 
-    // 2. overlaps of all pairs i < j of the chunk
+    // 2. overlaps of all ordered pairs (i, j) of the chunk: each thread writes along a row
     for (int p = threadIdx.x; p < nI * nI; p += THREADS) {
         const int i = p / nI, j = p - i * nI;
-        if (j <= i) continue;
+        if (j == i) continue;
         const uint32_t* x = bm + i * pitch;
         const uint32_t* y = bm + j * pitch;
         int cnt = 0;
         for (int w = 0; w < nwords; ++w) cnt += __popc(x[w] & y[w]);
-        const uint16_t c16 = (uint16_t)min(cnt, 65535);
-        ov[i * CH + j] = c16;
-        ov[j * CH + i] = c16;
+        ov[i * OVP + j] = (uint16_t)min(cnt, 65535);
     }
     __syncthreads();
 
@@ -107,7 +106,7 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
     {
         const int i = threadIdx.x >> 2, quarter = threadIdx.x & 3;
         const int j0 = quarter * (CH / 4);
-        const uint4* row = reinterpret_cast<const uint4*>(ov + i * CH + j0);
+        const uint4* row = reinterpret_cast<const uint4*>(ov + i * OVP + j0);
         for (int r = 0; r < ROUNDS; ++r) {
             if (threadIdx.x == 0) s_new[r & 1] = 0;
             uint32_t bk = 0;
@@ -207,7 +206,7 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
 
 static size_t plan_smem(int NB) {
     const int nwords = (NB + 31) >> 5;
-    return (size_t)CH * CH * sizeof(uint16_t) + (size_t)CH * (nwords | 1) * sizeof(uint32_t);
+    return (size_t)CH * OVP * sizeof(uint16_t) + (size_t)CH * (nwords | 1) * sizeof(uint32_t);
 }
 
 }  // namespace plan
