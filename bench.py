@@ -202,10 +202,13 @@ def merge_path_rooflines(usv, device, peak_gbs):
     zm2 = torch.empty_like(zm)
     ms_plan = time_call(lambda: usv.token_merge(z, metric, wl.grid, wl.merge_part, wl.r, out=zm2))
     ms_apply = time_call(lambda: usv.token_merge(z, None, wl.grid, wl.merge_part, wl.r, plan=plan, out=zm2))
+    usv.merge_plan_cache(plan)
+    ms_cached = time_call(lambda: usv.token_merge_apply(z, plan, out=zm2))
     ms_unm = time_call(lambda: usv.token_unmerge(zm, plan.pos, out=y))
     moved = z.numel() * 2 + zm.numel() * 2
     desc_bytes = metric.numel() * 2 + wl.B * wl.N * wl.d * 4
     return [
+        hbm_entry("usv_token_merge_apply", "merge_kernel (merged-source lists cached with the plan)", moved, ms_cached, peak_gbs),
         hbm_entry("usv_token_merge(metric=NULL)", "csr_count/scan/fill + merge_kernel", moved, ms_apply, peak_gbs,
                   "merge_kernel streams the bytes; the three CSR kernels before it are latency-bound"),
         hbm_entry("usv_token_unmerge", "unmerge_kernel", moved, ms_unm, peak_gbs),
@@ -526,8 +529,8 @@ def spawn_ranks(argv, n):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="wan1.3b_480p")
     ap.add_argument("--impl", default="usv", choices=["usv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -246,6 +246,23 @@ int usv_token_merge_local(int B, int N, int C, const void* x, int Hm, int dm, co
                           int r, void* x_merged, int32_t* dst_of, int32_t* pos, float* u_out,
                           int32_t* jstar_out, void* ws, size_t ws_bytes, void* stream);
 
+/* A plan applied to several tensors (Q, K and V of one layer, Fig. 2; hidden states): the lists of
+ * merged sources per destination that the merge needs can be built once and kept by the caller,
+ * so that every further merge with that plan is the streaming kernel alone (Eq. 12-14).
+ *   usv_merge_plan_cache: from dst_of / pos of a plan (as written by usv_token_merge) into `cache`
+ *     (device, 16-byte aligned, usv_merge_plan_cache_bytes(B, N) bytes, owned by the caller).
+ *   usv_token_merge_apply: x_merged = merge(x) with the cached plan; same result as
+ *     usv_token_merge(metric = NULL).  `cache` is not const: a destination with more than 32 merged
+ *     sources has its list sorted in place on first use.
+ * Grid, partition and r must be those the plan was made with.
+ */
+size_t usv_merge_plan_cache_bytes(int B, int N);
+int usv_merge_plan_cache(int B, int N, int T, int Hh, int W, int st, int sh, int sw, int r,
+                         const int32_t* dst_of, const int32_t* pos, void* cache, size_t cache_bytes,
+                         void* stream);
+int usv_token_merge_apply(int B, int N, int C, const void* x, int T, int Hh, int W, int st, int sh,
+                          int sw, int r, void* cache, void* x_merged, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * Token unmerge (Sec. 3.3, Eq. 15): y[b,n,:] = y_merged[b,pos[b,n],:].
  * y_merged: bf16 [B,Nm,C]; pos: int32 [B,N] with entries in [0,Nm); y: bf16 [B,N,C] (written).

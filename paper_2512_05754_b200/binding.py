@@ -47,7 +47,7 @@ def lib():
     L.usv_build_info.restype = ctypes.c_char_p
     L.usv_kernel_launches.restype = ctypes.c_ulonglong
     for name in ("usv_block_scores_workspace", "usv_sparse_attn_workspace",
-                 "usv_token_merge_workspace", "usv_unmerge_map_workspace"):
+                 "usv_token_merge_workspace", "usv_unmerge_map_workspace", "usv_merge_plan_cache_bytes"):
         getattr(L, name).restype = ctypes.c_size_t
     _lib = L
     return L
@@ -241,6 +241,7 @@ class MergePlan:
     r: int
     u: Optional[torch.Tensor] = None     # fp32 [B,N]
     jstar: Optional[torch.Tensor] = None  # int32 [B,N]
+    cache: Optional[torch.Tensor] = None  # merged-source lists of the plan (merge_plan_cache)
 
 
 def token_merge(x, metric, grid, part, r, plan=None, debug=False, window=None, out=None):
@@ -457,3 +458,36 @@ def sparse_attn_fwd_unmerge(q, k, v, sel, k_per_head, umap, N_full, N=None, scal
     if return_lse:
         res += (lse,)
     return res if len(res) > 1 else out
+
+
+def merge_plan_cache(plan):
+    """Builds (once) and returns the merged-source lists of a plan, kept on the plan object, so that
+    token_merge_apply is the streaming merge kernel alone."""
+    if plan.cache is None:
+        B, N = plan.pos.shape
+        T, Hh, W = plan.grid
+        st, sh, sw = plan.part
+        L = lib()
+        nbytes = L.usv_merge_plan_cache_bytes(B, N)
+        cache = torch.empty(int(nbytes), dtype=torch.uint8, device=plan.pos.device)
+        _check(L.usv_merge_plan_cache(B, N, T, Hh, W, st, sh, sw, int(plan.r), _ptr(plan.dst_of), _ptr(plan.pos),
+                                      _ptr(cache), ctypes.c_size_t(nbytes), _stream(plan.pos.device)),
+               "usv_merge_plan_cache")
+        plan.cache = cache
+    return plan.cache
+
+
+def token_merge_apply(x, plan, out=None):
+    """Merges x [B,N,C] (bf16) with a stored plan through its cached lists; same result as
+    token_merge(x, None, ..., plan=plan)."""
+    if x.dim() != 3 or x.dtype != torch.bfloat16 or not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x must be a contiguous CUDA bf16 [B,N,C] tensor")
+    B, N, C = x.shape
+    T, Hh, W = plan.grid
+    st, sh, sw = plan.part
+    cache = merge_plan_cache(plan)
+    if out is None:
+        out = torch.empty((B, N - plan.r, C), dtype=torch.bfloat16, device=x.device)
+    _check(lib().usv_token_merge_apply(B, N, C, _ptr(x), T, Hh, W, st, sh, sw, int(plan.r), _ptr(cache), _ptr(out),
+                                       _stream(x.device)), "usv_token_merge_apply")
+    return out

@@ -238,6 +238,10 @@ def test_merge_unmerge(usv, case):
         xm2, _ = usv.token_merge(x2.to(_dev()), None, grid, part, r, plan=plan)
         ref2 = oracle.round_to_bf16(oracle.merge_apply(x2, pg["dst_of"], pg["pos"], N - r))
         assert bf16_ulp_distance(bits(xm2), ref2).max() <= 1
+        # ... and so does the cached form of the plan (the streaming kernel alone), twice in a row
+        for _ in range(2):
+            xm3 = usv.token_merge_apply(x2.to(_dev()), plan)
+            assert torch.equal(xm3.view(torch.int16), xm2.view(torch.int16))
         # unmerge is an exact gather
         y = usv.token_unmerge(xm, plan.pos)
         assert np.array_equal(bits(y), oracle.unmerge(got, pg["pos"]))
