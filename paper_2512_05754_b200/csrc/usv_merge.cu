@@ -753,6 +753,91 @@ extern "C" int usv_token_unmerge(int B, int N, int Nm, int C, const void* y_merg
     return USV_OK;
 }
 
+// ---------------------------------------------------------------------------- stored plan
+// What merge_kernel needs of a plan, kept by the caller beside dst_of / pos so that applying the
+// plan to further tensors is the streaming kernel alone: row_src | off | csr | (cnt, cursor scratch),
+// each B * (N + 1) ints.
+namespace usv {
+static size_t cache_stride(int B, int N) { return align_up((size_t)B * ((size_t)N + 1) * sizeof(int32_t), 256); }
+
+static int fill_part(Part& p, int N, int T, int Hh, int W, int st, int sh, int sw, const char* who) {
+    if (T <= 0 || Hh <= 0 || W <= 0 || (int64_t)T * Hh * W != N)
+        return fail(USV_ERR_INVALID_ARG, "%s: T*Hh*W = %lld != N = %d", who, (long long)T * Hh * W, N);
+    if (st <= 0 || sh <= 0 || sw <= 0) return fail(USV_ERR_INVALID_ARG, "%s: partition sizes must be positive", who);
+    p.T = T; p.Hh = Hh; p.W = W; p.st = st; p.sh = sh; p.sw = sw;
+    p.nHy = ceil_div(Hh, sh); p.nWx = ceil_div(W, sw);
+    p.nB = ceil_div(T, st) * p.nHy * p.nWx;
+    return USV_OK;
+}
+}  // namespace usv
+
+extern "C" size_t usv_merge_plan_cache_bytes(int B, int N) {
+    if (B <= 0 || N <= 0) return 0;
+    return 5 * usv::cache_stride(B, N);
+}
+
+extern "C" int usv_merge_plan_cache(int B, int N, int T, int Hh, int W, int st, int sh, int sw, int r,
+                                    const int32_t* dst_of, const int32_t* pos, void* cache, size_t cache_bytes,
+                                    void* stream) {
+    using namespace usv;
+    if (B <= 0 || N <= 0) return fail(USV_ERR_INVALID_ARG, "merge_plan_cache: B,N must be positive");
+    if (B > 65535) return fail(USV_ERR_UNSUPPORTED, "merge_plan_cache: B > 65535");
+    Part p;
+    int rc = fill_part(p, N, T, Hh, W, st, sh, sw, "merge_plan_cache");
+    if (rc != USV_OK) return rc;
+    const int nA = N - p.nB;
+    if (r < 0 || r > nA) return fail(USV_ERR_INVALID_ARG, "merge_plan_cache: r=%d outside [0,%d]", r, nA);
+    if (dst_of == nullptr || pos == nullptr || cache == nullptr) return fail(USV_ERR_INVALID_ARG, "merge_plan_cache: null pointer");
+    if (!aligned16(cache)) return fail(USV_ERR_UNSUPPORTED, "merge_plan_cache: cache not 16-byte aligned");
+    if (cache_bytes < usv_merge_plan_cache_bytes(B, N))
+        return fail(USV_ERR_WORKSPACE, "merge_plan_cache: cache %zu < %zu", cache_bytes, usv_merge_plan_cache_bytes(B, N));
+    char* base = static_cast<char*>(cache);
+    const size_t cs = cache_stride(B, N);
+    int32_t* row_src = reinterpret_cast<int32_t*>(base);
+    int32_t* off = reinterpret_cast<int32_t*>(base + cs);
+    int32_t* csr = reinterpret_cast<int32_t*>(base + 2 * cs);
+    int32_t* cnt = reinterpret_cast<int32_t*>(base + 3 * cs);
+    int32_t* cursor = reinterpret_cast<int32_t*>(base + 4 * cs);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(cnt, 0, (size_t)B * p.nB * 4, s);
+    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "merge_plan_cache: memset: %s", cudaGetErrorString(e));
+    dim3 tg(ceil_div(N, 256), B);
+    csr_count_kernel<<<tg, 256, 0, s>>>(p, N, nA - r, dst_of, pos, cnt, row_src);
+    USV_CHECK_LAUNCH("csr_count_kernel");
+    csr_scan_kernel<<<dim3(ceil_div(p.nB, 1024), B), 1024, 0, s>>>(p.nB, cnt, off, cursor);
+    USV_CHECK_LAUNCH("csr_scan_kernel");
+    if (r > 0) {
+        csr_fill_kernel<<<tg, 256, 0, s>>>(p, N, r, dst_of, cursor, csr);
+        USV_CHECK_LAUNCH("csr_fill_kernel");
+    }
+    return USV_OK;
+}
+
+extern "C" int usv_token_merge_apply(int B, int N, int C, const void* x, int T, int Hh, int W, int st, int sh,
+                                     int sw, int r, void* cache, void* x_merged, void* stream) {
+    using namespace usv;
+    if (B <= 0 || N <= 0 || C <= 0) return fail(USV_ERR_INVALID_ARG, "token_merge_apply: B,N,C must be positive");
+    if (C % 8) return fail(USV_ERR_UNSUPPORTED, "token_merge_apply: C=%d not a multiple of 8", C);
+    Part p;
+    int rc = fill_part(p, N, T, Hh, W, st, sh, sw, "token_merge_apply");
+    if (rc != USV_OK) return rc;
+    const int nA = N - p.nB;
+    if (r < 0 || r > nA) return fail(USV_ERR_INVALID_ARG, "token_merge_apply: r=%d outside [0,%d]", r, nA);
+    if (x == nullptr || cache == nullptr || x_merged == nullptr) return fail(USV_ERR_INVALID_ARG, "token_merge_apply: null pointer");
+    if (!aligned16(x) || !aligned16(x_merged) || !aligned16(cache))
+        return fail(USV_ERR_UNSUPPORTED, "token_merge_apply: x/x_merged/cache not 16-byte aligned");
+    char* base = static_cast<char*>(cache);
+    const size_t cs = cache_stride(B, N);
+    const int Nm = N - r;
+    const int64_t rows = (int64_t)B * Nm;
+    merge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        p, N, C, nA - r, Nm, r, static_cast<const __nv_bfloat16*>(x), reinterpret_cast<const int32_t*>(base),
+        reinterpret_cast<const int32_t*>(base + cs), reinterpret_cast<int32_t*>(base + 2 * cs),
+        static_cast<__nv_bfloat16*>(x_merged), rows);
+    USV_CHECK_LAUNCH("merge_kernel");
+    return USV_OK;
+}
+
 extern "C" size_t usv_unmerge_map_workspace(int B, int Nm) {
     if (B <= 0 || Nm <= 0) return 0;
     return usv::WS_HEADER + 2 * usv::align_up((size_t)B * Nm * sizeof(int32_t), 256);
