@@ -13,9 +13,11 @@ namespace usv {
 
 namespace plan {
 
-constexpr int ROUNDS = 6;      // upper limit; the matching stops as soon as a round finds nothing new
+constexpr int ROUNDS = 5;      // upper limit; the matching stops as soon as a round finds nothing new
 constexpr int CH = 128;        // query blocks per chunk
 constexpr int THREADS = 4 * CH;
+// bitmap row pitch in 32-bit words: the smallest 4 x odd number that holds the row
+__host__ __device__ inline int plan_pitch(int nwords) { const int q = (nwords + 3) / 4; return 4 * (q | 1); }
 constexpr int OVP = CH + 8;     // row pitch of the overlap matrix (uint16): rows start 4 banks apart
 
 // One CTA per chunk of CH consecutive query blocks of one (batch, head).
@@ -37,7 +39,8 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
     const int NB = a.NB;
     const int NP = (NB + 1) >> 1;
     const int nwords = (NB + 31) >> 5;
-    const int pitch = nwords | 1;                       // odd row pitch: rows start in different banks
+    const int pitch = plan_pitch(nwords);               // row pitch in words: 4 x odd, so that 16-byte loads of
+                                                        // consecutive rows fall into different bank groups
     uint16_t* ov = reinterpret_cast<uint16_t*>(smem_u);            // [CH][OVP], rows 16-byte aligned
     uint32_t* bm = smem_u + CH * OVP / 2;                          // [CH][pitch]
     const int bh = blockIdx.y;
@@ -65,7 +68,7 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
     }
 
     // 1. bitmaps
-    for (int i = threadIdx.x; i < nI * pitch; i += THREADS) bm[i] = 0u;
+    for (int i = threadIdx.x; i < CH * pitch; i += THREADS) bm[i] = 0u;
     __syncthreads();
     const int32_t* sel = a.sel + ((int64_t)bh * NB + I0) * a.kmax;
     const int total = nI * kh;
@@ -89,15 +92,31 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
     for (int i = threadIdx.x; i < CH * OVP / 2; i += THREADS) smem_u[i] = 0u;   // overlaps of blocks past the end: 0
     __syncthreads();
 
-    // 2. overlaps of all ordered pairs (i, j) of the chunk: each thread writes along a row
-    for (int p = threadIdx.x; p < nI * nI; p += THREADS) {
-        const int i = p / nI, j = p - i * nI;
-        if (j == i) continue;
-        const uint32_t* x = bm + i * pitch;
-        const uint32_t* y = bm + j * pitch;
-        int cnt = 0;
-        for (int w = 0; w < nwords; ++w) cnt += __popc(x[w] & y[w]);
-        ov[i * OVP + j] = (uint16_t)min(cnt, 65535);
+    // 2. overlaps of all ordered pairs (i, j) of the chunk.  A thread takes four rows i against one
+    // row j, 128 bits of each at a time: the four i rows are the same for the whole warp (broadcast),
+    // consecutive lanes take consecutive j and write along a row.
+    {
+        const int nq = pitch / 4;
+        const int nIb = (nI + 3) / 4;
+        for (int p = threadIdx.x; p < nIb * nI; p += THREADS) {
+            const int ib = p / nI, j = p - ib * nI;
+            const uint4* y = reinterpret_cast<const uint4*>(bm + j * pitch);
+            const uint4* x = reinterpret_cast<const uint4*>(bm + ib * 4 * pitch);   // rows past nI are zero
+            int cnt[4] = {0, 0, 0, 0};
+            for (int w = 0; w < nq; ++w) {
+                const uint4 yv = y[w];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint4 xv = x[q * nq + w];
+                    cnt[q] += __popc(xv.x & yv.x) + __popc(xv.y & yv.y) + __popc(xv.z & yv.z) + __popc(xv.w & yv.w);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int i = ib * 4 + q;
+                if (i < nI && i != j) ov[i * OVP + j] = (uint16_t)min(cnt[q], 65535);
+            }
+        }
     }
     __syncthreads();
 
@@ -206,7 +225,7 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
 
 static size_t plan_smem(int NB) {
     const int nwords = (NB + 31) >> 5;
-    return (size_t)CH * OVP * sizeof(uint16_t) + (size_t)CH * (nwords | 1) * sizeof(uint32_t);
+    return (size_t)CH * OVP * sizeof(uint16_t) + (size_t)CH * plan_pitch(nwords) * sizeof(uint32_t);
 }
 
 }  // namespace plan
