@@ -20,7 +20,7 @@
 //                       destination rows stream through shared memory (TMA, 4 stages); warp 8 =
 //                       TMA producer, warps 9-10 = MMA issuers on alternate tiles, warps 0-3 / 4-7 =
 //                       two groups of one thread per source row, reading the 128 x 128 tiles of even /
-//                       odd index out of TMEM (a buffer each) and keeping the eight best (value,
+//                       odd index out of TMEM (three accumulator tiles in rotation) and keeping the eight best (value,
 //                       destination) inside the window of their running maximum, ascending destinations
 //   recheck_kernel      per source: the candidates inside the window in fp32 -> j*, u; sources
 //                       with a full window are listed
@@ -38,6 +38,8 @@ using namespace t5;
 
 constexpr int DM = 128;
 constexpr int STAGES = 4;
+constexpr int NBUF = 3;                                 // accumulator tiles in TMEM: the hand-over of a tile between
+                                                        // MMA issuer and epilogue takes longer than its MMAs
 constexpr uint32_t STAGE_BYTES = 128 * DM * 2;          // 32 KB: fp16 rows of a tile, [d-half][128 rows][128 B]
 constexpr int W_PROD = 8, W_MMA0 = 9;                   // warps 0-7: two epilogue warpgroups
 constexpr int NCAND = 8;                                // best approximate cosines kept per source and tile parity
@@ -47,13 +49,15 @@ constexpr uint32_t SM_SCR = SM_B + STAGES * STAGE_BYTES;   // float[32][256]: a 
 constexpr uint32_t SM_CV = SM_SCR + 32 * 256 * 4;          // float[NCAND][256]: candidate values per epilogue thread, descending
 constexpr uint32_t SM_CI = SM_CV + NCAND * 256 * 4;        // int[NCAND][256]: their destinations
 constexpr uint32_t SM_BAR = SM_CI + NCAND * 256 * 4;
-enum { B_AFULL = 0, B_BFULL = 1, B_BEMPTY = B_BFULL + STAGES, B_DFULL = B_BEMPTY + STAGES, B_DFREE = B_DFULL + 2,
-       B_COUNT = B_DFREE + 2 };
-constexpr uint32_t SM_MISC = SM_BAR + 8 * 16;
+enum { B_AFULL = 0, B_BFULL = 1, B_BEMPTY = B_BFULL + STAGES, B_DFULL = B_BEMPTY + STAGES, B_DFREE = B_DFULL + 2 * NBUF,
+       B_COUNT = B_DFREE + 2 * NBUF };
+static_assert(B_COUNT <= 32, "barrier area");
+constexpr uint32_t SM_MISC = SM_BAR + 8 * 32;
 constexpr uint32_t SM_TOTAL = SM_MISC + 64;
 constexpr size_t SMEM_BYTES = SM_TOTAL + 1024;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t TA = 0, TD = 128;                    // A rows (fp16) at 0; D buffers at 128 and 256
+constexpr uint32_t TA = 0, TD = 128;                    // A rows (fp16) at 0; D buffers at 128, 256 and 384
+static_assert(TD + NBUF * 128 <= TMEM_COLS, "TMEM budget");
 
 __global__ void __launch_bounds__(256)
 half_kernel(const float* __restrict__ mhat, MatchTcArgs m) {
@@ -125,7 +129,8 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.y;
     const int a0 = blockIdx.x * 128;
-    const int T = m.nB_pad / 128;   // destination tiles
+    const int T = m.nB_pad / 128;   // destination tiles, walked in the same order by every CTA (walking them
+                                    // in rotated orders, so that the CTAs ask for different L2 lines, was slower)
 
     if (threadIdx.x == 0) {
         mbar_init(bar(B_AFULL), 4);
@@ -133,7 +138,10 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
             mbar_init(bar(B_BFULL + s), 1);
             mbar_init(bar(B_BEMPTY + s), 1);
         }
-        for (int s = 0; s < 2; ++s) {
+        // Tile t uses accumulator t mod NBUF but the barriers t mod (2 NBUF): consecutive uses of an
+        // accumulator belong to different issuer warps and epilogue groups (t and t + NBUF differ in
+        // parity), and a waiter must see every phase of the barrier it waits on.
+        for (int s = 0; s < 2 * NBUF; ++s) {
             mbar_init(bar(B_DFULL + s), 1);
             mbar_init(bar(B_DFREE + s), 4);
         }
@@ -167,16 +175,16 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
         }
     } else if (warp == W_MMA0 || warp == W_MMA0 + 1) {
         // ===== two MMA issuers: warp 5 takes the even tiles, warp 6 the odd ones (each tile has its
-        // own B stage and D buffer), so that one warp's barrier waits fall under the other's MMAs =====
+        // own B stage and accumulator tile), so that one warp's barrier waits fall under the other's MMAs =====
         constexpr uint32_t IDESC = instr_desc_f16(128, 128, 0, 0);   // fp16 A (TMEM) x fp16 B (K-major) -> fp32
         const uint64_t bdesc0 = smem_desc(base + SM_B, 16, 1024);
         bool ok = mbar_wait(bar(B_AFULL), 0, s_abort, m.status, 0x20000);
         for (int t = warp - W_MMA0; ok && t < T; t += 2) {
             const int s = t % STAGES;
             const uint32_t ph = (t / STAGES) & 1;
-            const int buf = t & 1;
+            const int buf = t % NBUF;
             if (!mbar_wait_spin(bar(B_BFULL + s), ph, s_abort, m.status, 0x40000)) break;
-            if (t >= 2 && !mbar_wait_spin(bar(B_DFREE + buf), ((t - 2) >> 1) & 1, s_abort, m.status, 0x80000)) break;
+            if (t >= NBUF && !mbar_wait_spin(bar(B_DFREE + (t - NBUF) % (2 * NBUF)), ((t - NBUF) / (2 * NBUF)) & 1, s_abort, m.status, 0x80000)) break;
             fence_after();
             const uint64_t bd = bdesc0 + ((s * STAGE_BYTES) >> 4);
             const uint32_t d = tmem + TD + buf * 128;
@@ -185,13 +193,13 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
                 for (int ks = 0; ks < DM / 16; ++ks)
                     umma_ts(d, tmem + TA + ks * 8, bd + (((ks >> 2) * 16384 + (ks & 3) * 32) >> 4), IDESC, ks > 0);
                 umma_commit(bar(B_BEMPTY + s));
-                umma_commit(bar(B_DFULL + buf));
+                umma_commit(bar(B_DFULL + t % (2 * NBUF)));
             }
             __syncwarp();
         }
     } else {
         // ===== two warpgroups, one thread per source row in each: group e reads the tiles of parity e
-        // (D buffer e) and keeps its own candidates; the two lists meet in recheck_kernel =====
+        // (accumulator tile t mod NBUF) and keeps its own candidates; the two lists meet in recheck_kernel =====
         const int eg = warp >> 2;           // 0: even tiles, 1: odd tiles
         const int r = threadIdx.x & 127;    // TMEM lane = source row of the CTA
         const int a = a0 + r;
@@ -225,17 +233,18 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
         const float floor_v = m.floor_v[(int64_t)b * m.nA_pad + a];   // never above the row's approximate maximum
         bool ok = true;
         for (int t = eg; t < T; t += 2) {
-            if (!mbar_wait_spin(bar(B_DFULL + eg), (t >> 1) & 1, s_abort, m.status, 0x100000)) { ok = false; break; }
+            const int buf = t % NBUF;
+            if (!mbar_wait_spin(bar(B_DFULL + t % (2 * NBUF)), (t / (2 * NBUF)) & 1, s_abort, m.status, 0x100000)) { ok = false; break; }
             fence_after();
             const int nvalid = m.p.nB - t * 128;   // destinations of this tile that exist
             // the whole 128-column row in one go (four loads in flight, one wait), then the buffer goes back
             uint32_t sr[128];
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) tmem_ld32(lane_base + TD + eg * 128 + ch * 32, sr + ch * 32);
+            for (int ch = 0; ch < 4; ++ch) tmem_ld32(lane_base + TD + buf * 128 + ch * 32, sr + ch * 32);
             tmem_wait_ld();
             fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B_DFREE + eg));
+            if (lane == 0) mbar_arrive(bar(B_DFREE + t % (2 * NBUF)));
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
                 if (nvalid < (ch + 1) * 32) {   // only the chunks of the last tile that reach past the end (uniform)
@@ -273,13 +282,15 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
                         const float v = scr[j * 256];
                         if (v >= fmaxf(vmax, floor_v) - 2.0f * EPS && v > vlast) {
                             int pos = NCAND - 1;
-                            while (pos > 0 && v > cval[(pos - 1) * 256]) {     // strictly greater: a tie stays behind
+                            const int idx = t * 128 + ch * 32 + j;
+                            // descending cosine, then ascending destination
+                            while (pos > 0 && (v > cval[(pos - 1) * 256] || (v == cval[(pos - 1) * 256] && idx < cidx[(pos - 1) * 256]))) {
                                 cval[pos * 256] = cval[(pos - 1) * 256];
                                 cidx[pos * 256] = cidx[(pos - 1) * 256];
                                 --pos;
                             }
                             cval[pos * 256] = v;
-                            cidx[pos * 256] = t * 128 + ch * 32 + j;
+                            cidx[pos * 256] = idx;
                             vmax = cval[0];
                             vlast = cval[(NCAND - 1) * 256];
                         }
