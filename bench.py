@@ -65,20 +65,64 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and clock-event reasons while the timed region runs.
+
+    The timed region of the default run lasts tens of milliseconds, so the samples are read through
+    NVML from a thread of this process, one every millisecond or two (reads only; nothing is set);
+    `nvidia-smi -lms`, whose shortest period is longer than the region, is the fallback."""
     Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index):
-        self.gpu = gpu_index
+    def __init__(self, device):
+        self.device = device
         self.proc = None
         self.lines = []
+        self.samples = []          # (time, sm MHz, power W, reasons bit mask)
+        self.nvml = None
+        self.handle = None
+        self.stop_flag = False
+        self.thread = None
+        self.sm_max = None
+
+    def _nvml_open(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(self.device).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except TypeError:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            pynvml.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+            self.nvml = pynvml
+            return True
+        except Exception:
+            self.nvml = None
+            return False
+
+    def _poll(self):
+        nv, h = self.nvml, self.handle
+        while not self.stop_flag:
+            try:
+                self.samples.append((time.time(), float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)),
+                                     nv.nvmlDeviceGetPowerUsage(h) / 1000.0,
+                                     int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))))
+            except Exception:
+                break
+            time.sleep(0.001)
 
     def start(self):
+        if self._nvml_open():
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                ["nvidia-smi", "-i", str(self.device.index), "--query-gpu=" + self.Q,
                  "--format=csv,noheader,nounits", "-lms", "100"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
@@ -90,7 +134,25 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.time(), line.strip()))
 
+    def _stop_nvml(self, t0, t1):
+        nv = self.nvml
+        self.stop_flag = True
+        self.thread.join(timeout=2)
+        rows = [x for x in self.samples if t0 <= x[0] <= t1] or self.samples[-3:]
+        bits = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown,
+                "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown,
+                "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown,
+                "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap}
+        reasons = sorted(name for name, bit in bits.items() if any(x[3] & bit for x in rows))
+        return {"sm_mhz": float(np.median([x[1] for x in rows])) if rows else None,
+                "sm_min_mhz": float(min(x[1] for x in rows)) if rows else None,
+                "sm_max_mhz": self.sm_max,
+                "power_w": float(np.median([x[2] for x in rows])) if rows else None,
+                "samples": len(rows), "source": "nvml", "reasons": reasons}
+
     def stop(self, t0, t1):
+        if self.nvml is not None:
+            return self._stop_nvml(t0, t1)
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)
@@ -116,7 +178,7 @@ class ClockSampler:
         return {"sm_mhz": float(np.median(sm)) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None,
                 "power_w": float(np.median(power)) if power else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "source": "nvidia-smi", "reasons": sorted(reasons)}
 
 
 def flops(wl, N, k_per_head):
@@ -277,10 +339,10 @@ def run_usv(args, wl, rank, world, device):
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(device.index)
+    sampler = ClockSampler(device)
     if rank == 0:
         sampler.start()
-        time.sleep(0.25)
+        time.sleep(0.05)
     t_wall0 = time.time()
     e0, e1 = ev(), ev()
     barrier()
