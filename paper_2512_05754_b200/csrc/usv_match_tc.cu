@@ -245,6 +245,10 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
             fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(B_DFREE + t % (2 * NBUF)));
+            // The four chunk maxima first (three-input maxima on sixteen independent chains), and
+            // from them the tile's: most tiles lie below the window of the running maximum and are done
+            // here.  (The maximum only grows, so a destination below the window can never matter.)
+            float cm[4];
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
                 if (nvalid < (ch + 1) * 32) {   // only the chunks of the last tile that reach past the end (uniform)
@@ -252,10 +256,6 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
                     for (int j = 0; j < 32; ++j)
                         if (ch * 32 + j >= nvalid) sr[ch * 32 + j] = 0xff800000u;   // -inf: a destination that does not exist
                 }
-                // The chunk's maximum first (three-input maxima on four independent chains); only a
-                // chunk that reaches into the window of the running maximum is gone through element by
-                // element, in ascending order (the maximum only grows, so a destination below the
-                // window can never matter).
                 float c0 = max3(sr[ch * 32], sr[ch * 32 + 1], sr[ch * 32 + 2]);
                 float c1 = max3(sr[ch * 32 + 3], sr[ch * 32 + 4], sr[ch * 32 + 5]);
                 float c2 = max3(sr[ch * 32 + 6], sr[ch * 32 + 7], sr[ch * 32 + 8]);
@@ -269,30 +269,45 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
                 }
                 c0 = max3(__float_as_uint(c0), sr[ch * 32 + 28], sr[ch * 32 + 29]);
                 c1 = max3(__float_as_uint(c1), sr[ch * 32 + 30], sr[ch * 32 + 31]);
-                const float cm = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
-                if (cm >= fmaxf(vmax, floor_v) - 2.0f * EPS && cm > vlast) {
-                    // rare: the chunk goes through shared memory so that the insertion is ONE rolled
-                    // loop (unrolled over 128 register elements it is tens of KB of code, and the
-                    // kernel then waits on instruction fetch more than on anything else)
-                    float* scr = reinterpret_cast<float*>(sm + SM_SCR) + (threadIdx.x & 255);
+                cm[ch] = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
+            }
+            const float tm = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
+            if (tm >= fmaxf(vmax, floor_v) - 2.0f * EPS && tm > vlast) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) scr[j * 256] = __uint_as_float(sr[ch * 32 + j]);
+                for (int ch = 0; ch < 4; ++ch) {
+                    const float thr = fmaxf(vmax, floor_v) - 2.0f * EPS;
+                    if (cm[ch] >= thr && cm[ch] > vlast) {
+                        // Rare.  The chunk is parked in shared memory and a bit mask marks the elements
+                        // inside the window as it stands; only those are read back and inserted (one
+                        // short rolled loop: unrolled over the register elements the insertion is
+                        // tens of KB of code, and the kernel then waits on instruction fetch).
+                        float* scr = reinterpret_cast<float*>(sm + SM_SCR) + (threadIdx.x & 255);
+                        uint32_t mask = 0;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float v = __uint_as_float(sr[ch * 32 + j]);
+                            scr[j * 256] = v;
+                            if (v >= thr && v > vlast) mask |= 1u << j;
+                        }
 #pragma unroll 1
-                    for (int j = 0; j < 32; ++j) {
-                        const float v = scr[j * 256];
-                        if (v >= fmaxf(vmax, floor_v) - 2.0f * EPS && v > vlast) {
-                            int pos = NCAND - 1;
-                            const int idx = t * 128 + ch * 32 + j;
-                            // descending cosine, then ascending destination
-                            while (pos > 0 && (v > cval[(pos - 1) * 256] || (v == cval[(pos - 1) * 256] && idx < cidx[(pos - 1) * 256]))) {
-                                cval[pos * 256] = cval[(pos - 1) * 256];
-                                cidx[pos * 256] = cidx[(pos - 1) * 256];
-                                --pos;
+                        while (mask != 0) {
+                            const int j = __ffs(mask) - 1;
+                            mask &= mask - 1;
+                            const float v = scr[j * 256];
+                            if (v >= fmaxf(vmax, floor_v) - 2.0f * EPS && v > vlast) {
+                                int pos = NCAND - 1;
+                                const int idx = t * 128 + ch * 32 + j;
+                                // descending cosine, then ascending destination
+                                while (pos > 0 && (v > cval[(pos - 1) * 256] || (v == cval[(pos - 1) * 256] && idx < cidx[(pos - 1) * 256]))) {
+                                    cval[pos * 256] = cval[(pos - 1) * 256];
+                                    cidx[pos * 256] = cidx[(pos - 1) * 256];
+                                    --pos;
+                                }
+                                cval[pos * 256] = v;
+                                cidx[pos * 256] = idx;
+                                vmax = cval[0];
+                                vlast = cval[(NCAND - 1) * 256];
                             }
-                            cval[pos * 256] = v;
-                            cidx[pos * 256] = idx;
-                            vmax = cval[0];
-                            vlast = cval[(NCAND - 1) * 256];
                         }
                     }
                 }
