@@ -292,6 +292,44 @@ def test_matching_with_crowded_windows_dm128(usv):
         assert bf16_ulp_distance(bits(xm), ref).max() <= 1
 
 
+def test_matching_exact_ties_inside_the_candidate_lists_dm128(usv):
+    """dm = 128.  A few sources have three destinations that carry exactly their own descriptor
+    (cosine 1, equal to the last bit), far apart: in different 128-destination tiles, handled by
+    different epilogue groups of the matcher.  Three candidates fit its lists, so these sources
+    are settled by the fp32 re-check of the lists and not by the full scan: the lowest of the three
+    destinations must win (Eq. 9 with ties to the lowest index), and the rest of the plan must be
+    the oracle's."""
+    grid, part = (4, 12, 32), (1, 1, 2)                    # 1536 tokens, 768 destinations = 6 tiles
+    N = 1536
+    g = torch.Generator().manual_seed(91)
+    metric = torch.randn(N, 2, 128, generator=g)
+    is_dst = oracle.destination_mask(grid, part)
+    dst = np.nonzero(is_dst)[0]
+    src = np.nonzero(~is_dst)[0]
+    cases = {}
+    for i, a in enumerate(src[[3, 200, 411, 700]]):
+        trio = dst[[17 + 40 * i, 17 + 40 * i + 131, 17 + 40 * i + 390]]   # tiles t, t + 1, t + 3
+        for j in trio:
+            metric[j] = metric[a]
+        cases[int(a)] = int(trio.min())
+    metric = metric.unsqueeze(0).to(torch.bfloat16)
+    x = _rand_bf16((1, N, 64), 92)
+    for r in (0, 300, 768):
+        xm, plan = usv.token_merge(x.to(_dev()), metric.to(_dev()), grid, part, r, debug=True)
+        torch.cuda.synchronize()
+        assert usv.workspace_status() == 0
+        jstar = plan.jstar.cpu().numpy()
+        u = plan.u.cpu().numpy()
+        for a, jmin in cases.items():
+            assert jstar[0, a] == jmin, (a, jstar[0, a], jmin)
+            assert abs(u[0, a] - 1.0) < 1e-6
+        pg = dict(dst_of=plan.dst_of.cpu().numpy(), pos=plan.pos.cpu().numpy(), u=u, jstar=jstar)
+        stats = check_merge_plan(pg, metric, grid, part, r)
+        assert stats["jstar_differ"] == 0
+        ref = oracle.round_to_bf16(oracle.merge_apply(x, pg["dst_of"], pg["pos"], N - r))
+        assert bf16_ulp_distance(bits(xm), ref).max() <= 1
+
+
 # ---------------------------------------------------------------- argument validation on device
 
 def test_errors_leave_outputs_untouched(usv):
