@@ -78,6 +78,18 @@ def test_sequence_length_sweep(usv, name):
     _attention_parity(usv, q, k, v, wl.N, wl.k_per_head(), 24, 50 + wl.index)
 
 
+@pytest.mark.parametrize("grid", [(64, 64, 64), (64, 17, 241)])
+def test_longest_sequence_of_the_tensor_core_kernel_and_one_block_beyond(usv, grid):
+    """4096 key blocks (262 144 tokens) is the longest sequence the tcgen05 attention kernel takes
+    (its pairing plan keeps one bitmap row per query block in shared memory); with 4097 blocks the
+    same call runs the exact online-softmax kernel instead.  One head, 40 key blocks kept: rows of
+    4096 / 4097 scores through the selection kernel in full, attention on sampled query blocks."""
+    wl = ui.Workload("longest", 40, 1, 1, 128, grid, (1,), k_fixed=40)
+    assert wl.NB in (4096, 4097)
+    q, k, v = ui.make_qkv(wl, device=DEV, layout="bhnd")
+    _attention_parity(usv, q, k, v, wl.N, wl.k_per_head(), 6, 60 + wl.NB)
+
+
 def test_wan_14b_720p(usv):
     wl = ui.workload("wan14b_720p")
     q, k, v = ui.make_qkv(wl, device=DEV)
