@@ -147,7 +147,8 @@ int usv_select_blocks(int B, int H, int NBq, int NBk, const float* scores,
  * the other.  Results equal the per-block definition for finite inputs.  A NaN or infinity in K
  * or V inside a block that one query block of a pair selected can also reach the output rows of
  * its partner (0 * inf); blocks that neither selected are never read.  impl 1 keeps query blocks
- * fully separate.
+ * fully separate.  Sequences of more than 4096 key blocks (262 144 tokens), and d = 64, run the
+ * impl 1 kernel whatever impl says.
  */
 size_t usv_sparse_attn_workspace(int B, int H, int N, int d, int kmax);
 int usv_sparse_attn_fwd(int B, int H, int N, int d, const void* q, const usv_strides* sq,
