@@ -136,6 +136,45 @@ def test_keep_all_matches_dense_attention(usv):
         assert mx <= MAX_ABS and rl2 <= REL_L2, (impl, mx, rl2)
 
 
+@pytest.mark.parametrize("d", [128, 64])
+def test_query_blocks_without_keys_and_skipped_entries(usv, d):
+    """Degenerate selections: query blocks whose row holds no key block at all (defined output:
+    zeros, log-sum-exp 0), rows with -1 holes among their first k entries, a block with keys next
+    to a neighbour without any (whatever the kernel pairs them with), an odd number of key blocks
+    in a row, and the partial last block on both sides.  Every value against the oracle."""
+    B, H, N = 2, 3, 64 * 10 + 23                            # 11 blocks, the last with 23 tokens
+    NB, kmax, kph = 11, 4, [4, 3, 1]
+    wl = ui.Workload("degenerate%d" % d, 150 + d, B, H, d, (3, 13, 17), (100,))
+    q, k, v = ui.make_qkv(wl)
+    rng = np.random.default_rng(12)
+    sel = np.full((B, H, NB, kmax), -1, dtype=np.int32)
+    for b in range(B):
+        for h in range(H):
+            for i in range(NB):
+                sel[b, h, i, :kph[h]] = np.sort(rng.choice(NB, size=kph[h], replace=False))
+    sel[:, :, [0, 3, 4, 10], :] = -1                          # no key block at all
+    sel[0, 0, 5, 1] = -1                                      # holes inside the first k entries
+    sel[1, 1, 6, 0] = -1
+    sel[0, 0, 7, :] = [10, -1, -1, -1]                        # only the partial last key block
+    sel[1, 0, 9, :] = [2, 5, 10, -1]                          # an odd number of key blocks
+    for impl in (0, 1):
+        o, o32, lse = usv.sparse_attn_fwd(q.to(_dev()), k.to(_dev()), v.to(_dev()), torch.from_numpy(sel).to(_dev()),
+                                          kph, N=N, return_f32=True, return_lse=True, impl=impl)
+        torch.cuda.synchronize()
+        assert usv.workspace_status() == 0
+        o_ref, lse_ref = oracle.sparse_attn(q, k, v, N, sel, kph)
+        o_ref = o_ref.reshape(B, H, NB * 64, d)[:, :, :N]
+        lse_ref = lse_ref.reshape(B, H, NB * 64)[:, :, :N]
+        got = o32.cpu().numpy()
+        mx, rl2 = attn_errors(got, o_ref)
+        assert mx <= MAX_ABS and rl2 <= REL_L2, (impl, mx, rl2)
+        assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 2e-3
+        for i in (0, 3, 4):
+            assert not got[:, :, i * 64:(i + 1) * 64].any() and not o[:, :, i * 64:(i + 1) * 64].float().cpu().numpy().any()
+        assert not got[:, :, 640:].any()
+        assert torch.equal(o.cpu(), o32.to(torch.bfloat16).cpu())
+
+
 @pytest.mark.parametrize("kb,expect_fallback", [(20.0, False), (64.0, True)])
 def test_fixed_reference_range_and_exact_recomputation(usv, kb, expect_fallback):
     """The tcgen05 kernel fixes a row's softmax reference at its first key block.  Logits of a later
