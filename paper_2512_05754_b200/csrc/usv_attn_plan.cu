@@ -92,17 +92,34 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
     for (int i = threadIdx.x; i < CH * OVP / 2; i += THREADS) smem_u[i] = 0u;   // overlaps of blocks past the end: 0
     __syncthreads();
 
-    // 2. overlaps of all ordered pairs (i, j) of the chunk.  A thread takes four rows i against one
-    // row j, 128 bits of each at a time: the four i rows are the same for the whole warp (broadcast),
-    // consecutive lanes take consecutive j and write along a row.
+    // 2. overlaps of every two blocks of the chunk.  A thread takes four rows i (one row block)
+    // against one row j, 128 bits of each at a time: the four i rows are the same for most of a
+    // warp (broadcast), consecutive lanes take consecutive j.  The matrix is symmetric, so only
+    // j >= (first row of the block) is computed and written to both places.  In a full chunk the
+    // row blocks are folded in pairs (block f with block 31 - f: together always CH + 4 values of
+    // j), which gives every thread the same number of items.
     {
         const int nq = pitch / 4;
         const int nIb = (nI + 3) / 4;
-        for (int p = threadIdx.x; p < nIb * nI; p += THREADS) {
-            const int ib = p / nI, j = p - ib * nI;
+        const bool folded = nI == CH;
+        const int per = CH + 4;
+        const int items = folded ? (CH / 8) * per : nIb * nI;
+        for (int p = threadIdx.x; p < items; p += THREADS) {
+            int ib, j;
+            if (folded) {
+                const int f = p / per, t = p - f * per;
+                const int len = CH - 4 * f;            // values of j of block f
+                ib = t < len ? f : CH / 4 - 1 - f;
+                j = t < len ? 4 * f + t : 4 * ib + (t - len);
+            } else {
+                ib = p / nI;
+                j = p - ib * nI;
+                if (j < 4 * ib) continue;
+            }
             const uint4* y = reinterpret_cast<const uint4*>(bm + j * pitch);
             const uint4* x = reinterpret_cast<const uint4*>(bm + ib * 4 * pitch);   // rows past nI are zero
             int cnt[4] = {0, 0, 0, 0};
+#pragma unroll 2
             for (int w = 0; w < nq; ++w) {
                 const uint4 yv = y[w];
 #pragma unroll
@@ -114,7 +131,11 @@ pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ l
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const int i = ib * 4 + q;
-                if (i < nI && i != j) ov[i * OVP + j] = (uint16_t)min(cnt[q], 65535);
+                if (i < nI && i != j) {
+                    const uint16_t c = (uint16_t)min(cnt[q], 65535);
+                    ov[i * OVP + j] = c;
+                    if (j >= 4 * ib + 4) ov[j * OVP + i] = c;
+                }
             }
         }
     }
