@@ -46,9 +46,7 @@ constexpr int NCAND = 8;                                // best approximate cosi
 constexpr float EPS = 1.0e-3f;                          // bound on |approximate - exact cosine| (see above)
 constexpr uint32_t SM_B = 0;
 constexpr uint32_t SM_SCR = SM_B + STAGES * STAGE_BYTES;   // float[32][256]: a chunk of one row per epilogue thread
-constexpr uint32_t SM_CV = SM_SCR + 32 * 256 * 4;          // float[NCAND][256]: candidate values per epilogue thread, descending
-constexpr uint32_t SM_CI = SM_CV + NCAND * 256 * 4;        // int[NCAND][256]: their destinations
-constexpr uint32_t SM_BAR = SM_CI + NCAND * 256 * 4;
+constexpr uint32_t SM_BAR = SM_SCR + 32 * 256 * 4;
 enum { B_AFULL = 0, B_BFULL = 1, B_BEMPTY = B_BFULL + STAGES, B_DFULL = B_BEMPTY + STAGES, B_DFREE = B_DFULL + 2 * NBUF,
        B_COUNT = B_DFREE + 2 * NBUF };
 static_assert(B_COUNT <= 32, "barrier area");
@@ -222,13 +220,13 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(B_AFULL));
         }
-        // The NCAND largest approximate cosines so far (shared memory, one column per thread),
-        // descending; equal values keep the order of their destinations (ascending), so the lowest
-        // destination of a tie stands first.  vmax / vlast mirror the first and the last entry.
-        float* cval = reinterpret_cast<float*>(sm + SM_CV) + (threadIdx.x & 255);
-        int* cidx = reinterpret_cast<int*>(sm + SM_CI) + (threadIdx.x & 255);
+        // The NCAND largest approximate cosines so far (registers), descending; equal values keep
+        // the order of their destinations (ascending), so the lowest destination of a tie stands
+        // first.  vmax / vlast mirror the first and the last entry.
+        float cval[NCAND];
+        int cidx[NCAND];
 #pragma unroll
-        for (int c = 0; c < NCAND; ++c) { cval[c * 256] = -INFINITY; cidx[c * 256] = 0; }
+        for (int c = 0; c < NCAND; ++c) { cval[c] = -INFINITY; cidx[c] = 0; }
         float vmax = -INFINITY, vlast = -INFINITY;
         const float floor_v = m.floor_v[(int64_t)b * m.nA_pad + a];   // never above the row's approximate maximum
         bool ok = true;
@@ -295,18 +293,22 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
                             mask &= mask - 1;
                             const float v = scr[j * 256];
                             if (v >= fmaxf(vmax, floor_v) - 2.0f * EPS && v > vlast) {
-                                int pos = NCAND - 1;
                                 const int idx = t * 128 + ch * 32 + j;
-                                // descending cosine, then ascending destination
-                                while (pos > 0 && (v > cval[(pos - 1) * 256] || (v == cval[(pos - 1) * 256] && idx < cidx[(pos - 1) * 256]))) {
-                                    cval[pos * 256] = cval[(pos - 1) * 256];
-                                    cidx[pos * 256] = cidx[(pos - 1) * 256];
-                                    --pos;
+                                // descending cosine, then ascending destination: the entries the
+                                // new one beats move down one place, the last one drops out
+                                bool placed = false;
+#pragma unroll
+                                for (int pos = NCAND - 1; pos > 0; --pos) {
+                                    const bool up = v > cval[pos - 1] || (v == cval[pos - 1] && idx < cidx[pos - 1]);
+                                    if (!placed) {
+                                        cval[pos] = up ? cval[pos - 1] : v;
+                                        cidx[pos] = up ? cidx[pos - 1] : idx;
+                                    }
+                                    placed |= !up;
                                 }
-                                cval[pos * 256] = v;
-                                cidx[pos * 256] = idx;
+                                if (!placed) { cval[0] = v; cidx[0] = idx; }
                                 vmax = cval[0];
-                                vlast = cval[(NCAND - 1) * 256];
+                                vlast = cval[NCAND - 1];
                             }
                         }
                     }
@@ -317,8 +319,8 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
             const int64_t g4 = (((int64_t)b * m.nA + a) * 2 + eg) * NCAND;
 #pragma unroll
             for (int c = 0; c < NCAND; ++c) {
-                m.cand_v[g4 + c] = cval[c * 256];
-                m.cand_i[g4 + c] = cidx[c * 256];
+                m.cand_v[g4 + c] = cval[c];
+                m.cand_i[g4 + c] = cidx[c];
             }
         }
     }
