@@ -80,6 +80,7 @@ extern "C" int usv_workspace_status(void* ws, void* stream) {
 namespace usv {
 // One warp waits, with the library's own bounded wait, on a barrier that nothing ever arrives at.
 __global__ void wait_selftest_kernel(unsigned int* status, unsigned long long limit_ns) {
+    dep_sync();
     __shared__ __align__(8) unsigned long long bar_mem;
     __shared__ int abort_flag;
     const uint32_t bar = t5::smem_u32(&bar_mem);

@@ -224,6 +224,7 @@ __device__ __forceinline__ void attn_mma_block(const AttnArgs& a, const int work
 // One CTA per query block, or (list mode) a fixed grid whose CTAs walk a device-side work list.
 template <int D>
 __global__ void __launch_bounds__(128) attn_mma_kernel(const AttnArgs a) {
+    dep_sync();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (a.work_list == nullptr) {
         attn_mma_block<D>(a, blockIdx.x, smem_raw);
@@ -243,11 +244,11 @@ int launch_attn_mma(const AttnArgs& a, int d, cudaStream_t st) {
     if (d == 128) {
         cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)MmaSmem<128>::BYTES);
-        attn_mma_kernel<128><<<(unsigned)grid, 128, MmaSmem<128>::BYTES, st>>>(a);
+        launch_dep(attn_mma_kernel<128>, dim3((unsigned)grid), dim3(128), MmaSmem<128>::BYTES, st, a);
     } else {
         cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)MmaSmem<64>::BYTES);
-        attn_mma_kernel<64><<<(unsigned)grid, 128, MmaSmem<64>::BYTES, st>>>(a);
+        launch_dep(attn_mma_kernel<64>, dim3((unsigned)grid), dim3(128), MmaSmem<64>::BYTES, st, a);
     }
     USV_CHECK_LAUNCH("attn_mma_kernel");
     return USV_OK;

@@ -135,6 +135,7 @@ __device__ __forceinline__ const int* item_list(const int* hdr) {
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
+    dep_sync();
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -637,6 +638,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
 
 // Fused unmerge: query blocks the exact kernel recomputed sit in o; copy them to their tokens in y.
 __global__ void __launch_bounds__(128) scatter_fallback_kernel(const AttnArgs a) {
+    dep_sync();
     const int count = *a.fallback_count;
     const int NB = a.NB, N = a.N;
     for (int w = blockIdx.x; w < count; w += gridDim.x) {
@@ -661,7 +663,7 @@ __global__ void __launch_bounds__(128) scatter_fallback_kernel(const AttnArgs a)
 
 int launch_scatter_fallbacks(const AttnArgs& a, int d, cudaStream_t st) {
     (void)d;
-    pr::scatter_fallback_kernel<<<64, 128, 0, st>>>(a);
+    launch_dep(pr::scatter_fallback_kernel, dim3(64), dim3(128), 0, st, a);
     USV_CHECK_LAUNCH("scatter_fallback_kernel");
     return USV_OK;
 }
@@ -695,7 +697,7 @@ int launch_attn_pair(const AttnArgs& a, int d, cudaStream_t st) {
     if (fa.numRegs * (pr::NTHREADS / 32) < 16 * pr::REG_SOFT + 4 * pr::REG_EPI + 4 * pr::REG_SERVICE)
         return fail(USV_ERR_UNSUPPORTED, "sparse_attn: kernel built with %d registers per thread, the roles need %d per lane",
                     fa.numRegs, 16 * pr::REG_SOFT + 4 * pr::REG_EPI + 4 * pr::REG_SERVICE);
-    pr::attn_pair_kernel<<<grid, pr::NTHREADS, pr::SMEM_BYTES, st>>>(a, maps);
+    launch_dep(pr::attn_pair_kernel, dim3(grid), dim3(pr::NTHREADS), pr::SMEM_BYTES, st, a, maps);
     USV_CHECK_LAUNCH("attn_pair_kernel");
     return USV_OK;
 }

@@ -30,6 +30,7 @@ constexpr int OVP = CH + 8;     // row pitch of the overlap matrix (uint16): row
 //      selected it (one warp per pair)
 __global__ void __launch_bounds__(THREADS)
 pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ lists) {
+    dep_sync();
     extern __shared__ __align__(16) uint32_t smem_u[];
     __shared__ int16_t partner[CH];
     __shared__ int16_t best[CH];
@@ -281,7 +282,7 @@ int launch_pair_plan(AttnArgs& a, void* mem, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(plan::pair_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: plan smem attribute: %s", cudaGetErrorString(e));
     dim3 grid((a.NB + plan::CH - 1) / plan::CH, a.B * a.H);
-    plan::pair_plan_kernel<<<grid, plan::THREADS, smem, st>>>(a, pairs, lists);
+    launch_dep(plan::pair_plan_kernel, dim3(grid), dim3(plan::THREADS), smem, st, a, pairs, lists);
     USV_CHECK_LAUNCH("pair_plan_kernel");
     return USV_OK;
 }

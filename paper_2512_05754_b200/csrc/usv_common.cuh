@@ -36,6 +36,33 @@ void note_launch();
             return usv::fail(USV_ERR_CUDA, "%s: %s", (what), cudaGetErrorString(e__));      \
     } while (0)
 
+// ---- launches ----------------------------------------------------------------------------
+// The kernels of the library are launched with programmatic stream serialization: the CTAs of
+// a kernel may be scheduled while the kernel before it in the stream is still running (that
+// kernel says so in its first instruction), and they wait for that kernel's completion, and
+// the visibility of its writes, in dep_sync(), the first statement of every kernel.  What is
+// saved is the launch latency between dependent kernels, 2-3 us each: a tenth of a merge +
+// attention step with its 19 small kernels.  Nothing is read or written before dep_sync().
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dep(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+__device__ __forceinline__ void dep_sync() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- device helpers -------------------------------------------------------------------
 
 __device__ __forceinline__ void bf16x8_to_float(const uint4& v, float* f) {

@@ -24,6 +24,7 @@ namespace usv {
 //   whole cubes before its cube inside that row, then its rank inside its own (possibly cut) cube.
 __global__ void __launch_bounds__(256) cube_order_kernel(int T, int Hh, int W, int ct, int ch, int cw,
                                                          int32_t* __restrict__ perm, int32_t* __restrict__ inv) {
+    dep_sync();
     const int n = blockIdx.x * 256 + threadIdx.x;
     if (n >= T * Hh * W) return;
     const int x = n % W, y = (n / W) % Hh, t = n / (W * Hh);
@@ -39,6 +40,7 @@ __global__ void __launch_bounds__(256) cube_order_kernel(int T, int Hh, int W, i
 
 __global__ void __launch_bounds__(256) force_own_block_kernel(float* __restrict__ scores, int NBq, int NBk,
                                                               int64_t total, uint32_t value_bits) {
+    dep_sync();
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;   // (b, h, I) flattened
     if (i >= total) return;
     const int I = (int)(i % NBq);
@@ -59,6 +61,7 @@ struct CombineArgs {
 // o = (e^lse1 o1 + e^lse2 o2) / (e^lse1 + e^lse2), one warp per (b, h, n) row, D / 32 elements per lane.
 template <int D, bool F32IN>
 __global__ void __launch_bounds__(256) combine_kernel(const CombineArgs a) {
+    dep_sync();
     constexpr int EPL = D / 32;   // 4 or 2
     const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (row >= a.rows) return;
@@ -129,7 +132,7 @@ extern "C" int usv_cube_order(int T, int Hh, int W, int ct, int ch, int cw, int3
     if ((int64_t)T * Hh * W > 2147483647LL) return fail(USV_ERR_UNSUPPORTED, "cube_order: more than 2^31-1 tokens");
     if (perm == nullptr) return fail(USV_ERR_INVALID_ARG, "cube_order: null pointer");
     const int N = T * Hh * W;
-    cube_order_kernel<<<ceil_div(N, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(T, Hh, W, ct, ch, cw, perm, inv);
+    launch_dep(cube_order_kernel, dim3(ceil_div(N, 256)), dim3(256), 0, static_cast<cudaStream_t>(stream), T, Hh, W, ct, ch, cw, perm, inv);
     USV_CHECK_LAUNCH("cube_order_kernel");
     return USV_OK;
 }
@@ -140,7 +143,7 @@ static int set_own_block(const char* who, int B, int H, int NBq, int NBk, float*
     if (scores == nullptr) return fail(USV_ERR_INVALID_ARG, "%s: null pointer", who);
     const int64_t total = (int64_t)B * H * NBq;
     if ((total + 255) / 256 > 2147483647LL) return fail(USV_ERR_UNSUPPORTED, "%s: too many rows", who);
-    force_own_block_kernel<<<(unsigned)((total + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    launch_dep(force_own_block_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, static_cast<cudaStream_t>(stream), 
         scores, NBq, NBk, total, bits);
     USV_CHECK_LAUNCH("force_own_block_kernel");
     return USV_OK;
@@ -177,11 +180,11 @@ extern "C" int usv_attn_combine(int B, int H, int N, int d, const void* o1, cons
     if (blocks > 2147483647LL) return fail(USV_ERR_UNSUPPORTED, "attn_combine: too many rows");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (d == 128) {
-        if (inputs_f32) combine_kernel<128, true><<<(unsigned)blocks, 256, 0, st>>>(a);
-        else combine_kernel<128, false><<<(unsigned)blocks, 256, 0, st>>>(a);
+        if (inputs_f32) launch_dep((combine_kernel<128, true>), dim3((unsigned)blocks), dim3(256), 0, st, a);
+        else launch_dep((combine_kernel<128, false>), dim3((unsigned)blocks), dim3(256), 0, st, a);
     } else {
-        if (inputs_f32) combine_kernel<64, true><<<(unsigned)blocks, 256, 0, st>>>(a);
-        else combine_kernel<64, false><<<(unsigned)blocks, 256, 0, st>>>(a);
+        if (inputs_f32) launch_dep((combine_kernel<64, true>), dim3((unsigned)blocks), dim3(256), 0, st, a);
+        else launch_dep((combine_kernel<64, false>), dim3((unsigned)blocks), dim3(256), 0, st, a);
     }
     USV_CHECK_LAUNCH("combine_kernel");
     return USV_OK;

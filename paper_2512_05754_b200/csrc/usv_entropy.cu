@@ -19,6 +19,7 @@ namespace usv {
 
 template <int D>
 __global__ void __launch_bounds__(128) key_marginal_kernel(const MargArgs a) {
+    dep_sync();
     constexpr int LD = MmaSmem<D>::LD;
     constexpr int TILE = MmaSmem<D>::TILE;
     constexpr int KT = D / 16;
@@ -118,6 +119,7 @@ __global__ void __launch_bounds__(128) key_marginal_kernel(const MargArgs a) {
 
 // one CTA per batch element
 __global__ void __launch_bounds__(1024) entropy_kernel(const float* __restrict__ marg, int N, float* __restrict__ h) {
+    dep_sync();
     __shared__ float red[32];
     const float* m = marg + (int64_t)blockIdx.x * N;
     float s = 0.f;
@@ -183,10 +185,10 @@ extern "C" int usv_attn_entropy(int B, int H, int N, int d, const void* q, const
     } else {
         const size_t smem = (size_t)3 * MmaSmem<64>::TILE * sizeof(__nv_bfloat16);
         cudaFuncSetAttribute(key_marginal_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        key_marginal_kernel<64><<<(unsigned)grid, 128, smem, st>>>(a);
+        launch_dep(key_marginal_kernel<64>, dim3((unsigned)grid), dim3(128), smem, st, a);
     }
     if (d != 128) USV_CHECK_LAUNCH("key_marginal_kernel");
-    entropy_kernel<<<B, 1024, 0, st>>>(key_marginal, N, entropy);
+    launch_dep(entropy_kernel, dim3(B), dim3(1024), 0, st, key_marginal, N, entropy);
     USV_CHECK_LAUNCH("entropy_kernel");
     return USV_OK;
 }

@@ -52,6 +52,7 @@ struct Maps {
 
 __global__ void __launch_bounds__(NTHREADS, 2)
 marginal_tc_kernel(const MargArgs a, const __grid_constant__ Maps maps) {
+    dep_sync();
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -199,7 +200,7 @@ int launch_marginal_tc(const MargArgs& a, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(et::marginal_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)et::SMEM_BYTES);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "attn_entropy: smem attribute: %s", cudaGetErrorString(e));
-    et::marginal_tc_kernel<<<(unsigned)grid, et::NTHREADS, et::SMEM_BYTES, st>>>(a, maps);
+    launch_dep(et::marginal_tc_kernel, dim3((unsigned)grid), dim3(et::NTHREADS), et::SMEM_BYTES, st, a, maps);
     USV_CHECK_LAUNCH("marginal_tc_kernel");
     return USV_OK;
 }

@@ -59,6 +59,7 @@ static_assert(TD + NBUF * 128 <= TMEM_COLS, "TMEM budget");
 
 __global__ void __launch_bounds__(256)
 half_kernel(const float* __restrict__ mhat, MatchTcArgs m) {
+    dep_sync();
     // one warp per output row (4 floats per lane)
     const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
@@ -117,6 +118,7 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 
 __global__ void __launch_bounds__(352, 1)
 match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
+    dep_sync();
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -344,6 +346,7 @@ match_tc_kernel(const MatchTcArgs m, const __grid_constant__ Maps maps) {
 // appended to the list of the exact scan.
 __global__ void __launch_bounds__(256)
 recheck_kernel(const float* __restrict__ mhat, MatchTcArgs m) {
+    dep_sync();
     const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (gw >= (int64_t)m.B * m.nA) return;
@@ -390,6 +393,7 @@ constexpr int EX_CHUNK = 256;
 
 __global__ void __launch_bounds__(256)
 match_exact_kernel(const float* __restrict__ mhat, MatchTcArgs m) {
+    dep_sync();
     __shared__ unsigned long long s_key[8];
     const int count = *m.exact_count;
     const int nchunks = (m.p.nB + EX_CHUNK - 1) / EX_CHUNK;
@@ -436,6 +440,7 @@ match_exact_kernel(const float* __restrict__ mhat, MatchTcArgs m) {
 
 __global__ void __launch_bounds__(256)
 match_exact_finish_kernel(MatchTcArgs m) {
+    dep_sync();
     const int count = *m.exact_count;
     for (int w = blockIdx.x * 256 + threadIdx.x; w < count; w += gridDim.x * 256) {
         const unsigned long long key = m.exact_best[w];
@@ -499,7 +504,7 @@ int launch_match_tc(const float* mhat, const Part& p, int B, int N, int nA, cons
     cudaError_t e = cudaMemsetAsync(m.exact_count, 0, 256 + 2 * list_bytes(B, N), st);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: memset: %s", cudaGetErrorString(e));
     const int64_t rows = (int64_t)B * (m.nA_pad + m.nB_pad);
-    mt::half_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(mhat, m);
+    launch_dep(mt::half_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, st, mhat, m);
     USV_CHECK_LAUNCH("half_kernel");
     mt::Maps maps;
     int rc;
@@ -507,14 +512,14 @@ int launch_match_tc(const float* mhat, const Part& p, int B, int N, int nA, cons
     e = cudaFuncSetAttribute(mt::match_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mt::SMEM_BYTES);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: smem attribute: %s", cudaGetErrorString(e));
     dim3 grid(m.nA_pad / 128, B);
-    mt::match_tc_kernel<<<grid, 352, mt::SMEM_BYTES, st>>>(m, maps);
+    launch_dep(mt::match_tc_kernel, dim3(grid), dim3(352), mt::SMEM_BYTES, st, m, maps);
     USV_CHECK_LAUNCH("match_tc_kernel");
     const int64_t srcs = (int64_t)B * nA;
-    mt::recheck_kernel<<<(unsigned)((srcs + 7) / 8), 256, 0, st>>>(mhat, m);
+    launch_dep(mt::recheck_kernel, dim3((unsigned)((srcs + 7) / 8)), dim3(256), 0, st, mhat, m);
     USV_CHECK_LAUNCH("recheck_kernel");
-    mt::match_exact_kernel<<<1184, 256, 0, st>>>(mhat, m);
+    launch_dep(mt::match_exact_kernel, dim3(1184), dim3(256), 0, st, mhat, m);
     USV_CHECK_LAUNCH("match_exact_kernel");
-    mt::match_exact_finish_kernel<<<8, 256, 0, st>>>(m);
+    launch_dep(mt::match_exact_finish_kernel, dim3(8), dim3(256), 0, st, m);
     USV_CHECK_LAUNCH("match_exact_finish_kernel");
     return USV_OK;
 }

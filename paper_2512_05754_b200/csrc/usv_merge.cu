@@ -23,6 +23,7 @@ template <int DM>
 __global__ void __launch_bounds__(256) desc_kernel(const __nv_bfloat16* __restrict__ metric,
                                                    float* __restrict__ mhat, int64_t tokens,
                                                    int Hm) {
+    dep_sync();
     constexpr int LPH = DM / 8;    // lanes per head row
     constexpr int HPW = 32 / LPH;  // heads handled at once
     const int64_t tok = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -81,6 +82,7 @@ __device__ __forceinline__ int block_scan_1024(int v, int* scratch, int* total) 
 // its token index minus the number of destinations before it, which the partition gives in
 // closed form, so every token is handled independently.
 __global__ void __launch_bounds__(256) src_list_kernel(Part p, int N, int32_t* __restrict__ src_idx) {
+    dep_sync();
     const int n = blockIdx.x * 256 + threadIdx.x;
     if (n >= N || p.is_dst(n)) return;
     const int x = n % p.W, y = (n / p.W) % p.Hh, t = n / (p.W * p.Hh);
@@ -103,6 +105,7 @@ __global__ void __launch_bounds__(256) match_kernel(const float* __restrict__ mh
                                                     int nA, const int32_t* __restrict__ src_idx,
                                                     int32_t* __restrict__ jstar_s,
                                                     float* __restrict__ u_s) {
+    dep_sync();
     constexpr int TK = 32;
     __shared__ __align__(16) float As[DM][64 + 4];
     __shared__ __align__(16) float Bs[TK][64 + 4];
@@ -189,6 +192,7 @@ __global__ void __launch_bounds__(256) match_kernel(const float* __restrict__ mh
 // (Eq. 10 with ties to the lowest index), for 0 < r < nA.  One CTA per batch element.
 __global__ void __launch_bounds__(1024) plan_select_kernel(int nA, int r, const float* __restrict__ u_s,
                                                            int2* __restrict__ tsel) {
+    dep_sync();
     __shared__ int hist[256];
     __shared__ uint32_t s_prefix;
     __shared__ int s_remaining;
@@ -261,6 +265,7 @@ __global__ void __launch_bounds__(1024) plan_assign_kernel(Part p, int N, int nA
                                                            int32_t* __restrict__ pos,
                                                            float* __restrict__ u_out,
                                                            int32_t* __restrict__ jstar_out) {
+    dep_sync();
     __shared__ int scratch[33];
     const int b = blockIdx.y;
     const float* u = u_s + (int64_t)b * nA;
@@ -326,6 +331,7 @@ __global__ void __launch_bounds__(256) csr_count_kernel(Part p, int N, int nU,
                                                         const int32_t* __restrict__ pos,
                                                         int32_t* __restrict__ cnt,
                                                         int32_t* __restrict__ row_src) {
+    dep_sync();
     const int b = blockIdx.y;
     const int n = blockIdx.x * 256 + threadIdx.x;
     if (n >= N) return;
@@ -339,6 +345,7 @@ __global__ void __launch_bounds__(256) csr_count_kernel(Part p, int N, int nU,
 __global__ void __launch_bounds__(1024) csr_scan_kernel(int nB, const int32_t* __restrict__ cnt,
                                                         int32_t* __restrict__ off,
                                                         int32_t* __restrict__ cursor) {
+    dep_sync();
     __shared__ int scratch[33];
     const int b = blockIdx.y;
     const int o0 = blockIdx.x * 1024;
@@ -361,6 +368,7 @@ __global__ void __launch_bounds__(256) csr_fill_kernel(Part p, int N, int r,
                                                        const int32_t* __restrict__ dst_of,
                                                        int32_t* __restrict__ cursor,
                                                        int32_t* __restrict__ csr) {
+    dep_sync();
     const int b = blockIdx.y;
     const int n = blockIdx.x * 256 + threadIdx.x;
     if (n >= N) return;
@@ -381,6 +389,7 @@ __global__ void __launch_bounds__(256) match_local_kernel(const float* __restric
                                                           int wt, int wh, int ww,
                                                           const int32_t* __restrict__ src_idx,
                                                           int32_t* __restrict__ jstar_s, float* __restrict__ u_s) {
+    dep_sync();
     constexpr int V = DM / 32;   // floats per lane
     const int a = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (a >= nA) return;
@@ -422,6 +431,7 @@ __global__ void __launch_bounds__(256) merge_kernel(Part p, int N, int C, int nU
                                                     const int32_t* __restrict__ off,
                                                     int32_t* __restrict__ csr,
                                                     __nv_bfloat16* __restrict__ out, int64_t rows) {
+    dep_sync();
     const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (gw >= rows) return;
     const int lane = threadIdx.x & 31;
@@ -565,6 +575,7 @@ __global__ void __launch_bounds__(256) unmerge_kernel(int N, int Nm, int C,
                                                       const __nv_bfloat16* __restrict__ ym,
                                                       const int32_t* __restrict__ pos,
                                                       __nv_bfloat16* __restrict__ y, int64_t rows) {
+    dep_sync();
     const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (gw >= rows) return;
     const int lane = threadIdx.x & 31;
@@ -581,6 +592,7 @@ __global__ void __launch_bounds__(256) unmerge_kernel(int N, int Nm, int C,
 // merged row; the order inside a row is irrelevant, every token of a row receives the same values).
 __global__ void __launch_bounds__(256) inv_count_kernel(int N, int Nm, const int32_t* __restrict__ pos,
                                                         int32_t* __restrict__ cnt) {
+    dep_sync();
     const int b = blockIdx.y;
     const int n = blockIdx.x * 256 + threadIdx.x;
     if (n >= N) return;
@@ -590,6 +602,7 @@ __global__ void __launch_bounds__(256) inv_count_kernel(int N, int Nm, const int
 
 __global__ void __launch_bounds__(256) inv_fill_kernel(int N, int Nm, const int32_t* __restrict__ pos,
                                                        int32_t* __restrict__ cursor, int32_t* __restrict__ inv_idx) {
+    dep_sync();
     const int b = blockIdx.y;
     const int n = blockIdx.x * 256 + threadIdx.x;
     if (n >= N) return;
@@ -681,16 +694,16 @@ static int token_merge_impl(int B, int N, int C, const void* x, int Hm, int dm,
     if (metric != nullptr) {
         const int64_t tokens = (int64_t)B * N;
         const unsigned dg = (unsigned)((tokens + 7) / 8);
-        if (dm == 128) desc_kernel<128><<<dg, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(metric), mhat, tokens, Hm);
-        else desc_kernel<64><<<dg, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(metric), mhat, tokens, Hm);
+        if (dm == 128) launch_dep(desc_kernel<128>, dim3(dg), dim3(256), 0, s, static_cast<const __nv_bfloat16*>(metric), mhat, tokens, Hm);
+        else launch_dep(desc_kernel<64>, dim3(dg), dim3(256), 0, s, static_cast<const __nv_bfloat16*>(metric), mhat, tokens, Hm);
         USV_CHECK_LAUNCH("desc_kernel");
         if (nA > 0) {
-            src_list_kernel<<<ceil_div(N, 256), 256, 0, s>>>(p, N, src_idx);
+            launch_dep(src_list_kernel, dim3(ceil_div(N, 256)), dim3(256), 0, s, p, N, src_idx);
             USV_CHECK_LAUNCH("src_list_kernel");
             if (win != nullptr) {
                 dim3 lg(ceil_div(nA, 8), B);
-                if (dm == 128) match_local_kernel<128><<<lg, 256, 0, s>>>(mhat, p, N, nA, win[0], win[1], win[2], src_idx, jstar_s, u_s);
-                else match_local_kernel<64><<<lg, 256, 0, s>>>(mhat, p, N, nA, win[0], win[1], win[2], src_idx, jstar_s, u_s);
+                if (dm == 128) launch_dep(match_local_kernel<128>, dim3(lg), dim3(256), 0, s, mhat, p, N, nA, win[0], win[1], win[2], src_idx, jstar_s, u_s);
+                else launch_dep(match_local_kernel<64>, dim3(lg), dim3(256), 0, s, mhat, p, N, nA, win[0], win[1], win[2], src_idx, jstar_s, u_s);
                 USV_CHECK_LAUNCH("match_local_kernel");
             } else if (dm == 128) {
                 // tensor cores: split-bf16 cosines (usv_match_tc.cu)
@@ -699,36 +712,36 @@ static int token_merge_impl(int B, int N, int C, const void* x, int Hm, int dm,
                 if (rc != USV_OK) return rc;
             } else {
                 dim3 mg(ceil_div(nA, 64), B);
-                match_kernel<64><<<mg, 256, 0, s>>>(mhat, p, N, nA, src_idx, jstar_s, u_s);
+                launch_dep(match_kernel<64>, dim3(mg), dim3(256), 0, s, mhat, p, N, nA, src_idx, jstar_s, u_s);
                 USV_CHECK_LAUNCH("match_kernel");
             }
         }
         const int2* tsel = nullptr;
         if (r > 0 && r < nA) {
             int2* tsel_w = reinterpret_cast<int2*>(base + L.tsel);
-            plan_select_kernel<<<B, 1024, 0, s>>>(nA, r, u_s, tsel_w);
+            launch_dep(plan_select_kernel, dim3(B), dim3(1024), 0, s, nA, r, u_s, tsel_w);
             USV_CHECK_LAUNCH("plan_select_kernel");
             tsel = tsel_w;
         }
         // r = nA: every key is above 0; r = 0: no key is above or equal to the largest one
         dim3 pg(ceil_div(nA > p.nB ? nA : p.nB, 1024), B);
-        plan_assign_kernel<<<pg, 1024, 0, s>>>(p, N, nA, r, r == nA ? 0u : 0xffffffffu, 0, tsel, src_idx, jstar_s, u_s,
+        launch_dep(plan_assign_kernel, dim3(pg), dim3(1024), 0, s, p, N, nA, r, r == nA ? 0u : 0xffffffffu, 0, tsel, src_idx, jstar_s, u_s,
                                                dst_of, pos, u_out, jstar_out);
         USV_CHECK_LAUNCH("plan_assign_kernel");
     }
     cudaError_t e = cudaMemsetAsync(cnt, 0, (size_t)B * p.nB * 4, s);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: memset: %s", cudaGetErrorString(e));
     dim3 tg(ceil_div(N, 256), B);
-    csr_count_kernel<<<tg, 256, 0, s>>>(p, N, nU, dst_of, pos, cnt, row_src);
+    launch_dep(csr_count_kernel, dim3(tg), dim3(256), 0, s, p, N, nU, dst_of, pos, cnt, row_src);
     USV_CHECK_LAUNCH("csr_count_kernel");
-    csr_scan_kernel<<<dim3(ceil_div(p.nB, 1024), B), 1024, 0, s>>>(p.nB, cnt, off, cursor);
+    launch_dep(csr_scan_kernel, dim3(dim3(ceil_div(p.nB, 1024), B)), dim3(1024), 0, s, p.nB, cnt, off, cursor);
     USV_CHECK_LAUNCH("csr_scan_kernel");
     if (r > 0) {
-        csr_fill_kernel<<<tg, 256, 0, s>>>(p, N, r, dst_of, cursor, csr);
+        launch_dep(csr_fill_kernel, dim3(tg), dim3(256), 0, s, p, N, r, dst_of, cursor, csr);
         USV_CHECK_LAUNCH("csr_fill_kernel");
     }
     const int64_t rows = (int64_t)B * Nm;
-    merge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, s>>>(
+    launch_dep(merge_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, s, 
         p, N, C, nU, Nm, r, static_cast<const __nv_bfloat16*>(x), row_src, off, csr,
         static_cast<__nv_bfloat16*>(x_merged), rows);
     USV_CHECK_LAUNCH("merge_kernel");
@@ -746,7 +759,7 @@ extern "C" int usv_token_unmerge(int B, int N, int Nm, int C, const void* y_merg
     if (!aligned16(y_merged) || !aligned16(y))
         return fail(USV_ERR_UNSUPPORTED, "token_unmerge: y_merged/y not 16-byte aligned");
     const int64_t rows = (int64_t)B * N;
-    unmerge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    launch_dep(unmerge_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, static_cast<cudaStream_t>(stream), 
         N, Nm, C, static_cast<const __nv_bfloat16*>(y_merged), pos,
         static_cast<__nv_bfloat16*>(y), rows);
     USV_CHECK_LAUNCH("unmerge_kernel");
@@ -802,12 +815,12 @@ extern "C" int usv_merge_plan_cache(int B, int N, int T, int Hh, int W, int st, 
     cudaError_t e = cudaMemsetAsync(cnt, 0, (size_t)B * p.nB * 4, s);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "merge_plan_cache: memset: %s", cudaGetErrorString(e));
     dim3 tg(ceil_div(N, 256), B);
-    csr_count_kernel<<<tg, 256, 0, s>>>(p, N, nA - r, dst_of, pos, cnt, row_src);
+    launch_dep(csr_count_kernel, dim3(tg), dim3(256), 0, s, p, N, nA - r, dst_of, pos, cnt, row_src);
     USV_CHECK_LAUNCH("csr_count_kernel");
-    csr_scan_kernel<<<dim3(ceil_div(p.nB, 1024), B), 1024, 0, s>>>(p.nB, cnt, off, cursor);
+    launch_dep(csr_scan_kernel, dim3(dim3(ceil_div(p.nB, 1024), B)), dim3(1024), 0, s, p.nB, cnt, off, cursor);
     USV_CHECK_LAUNCH("csr_scan_kernel");
     if (r > 0) {
-        csr_fill_kernel<<<tg, 256, 0, s>>>(p, N, r, dst_of, cursor, csr);
+        launch_dep(csr_fill_kernel, dim3(tg), dim3(256), 0, s, p, N, r, dst_of, cursor, csr);
         USV_CHECK_LAUNCH("csr_fill_kernel");
     }
     return USV_OK;
@@ -830,7 +843,7 @@ extern "C" int usv_token_merge_apply(int B, int N, int C, const void* x, int T, 
     const size_t cs = cache_stride(B, N);
     const int Nm = N - r;
     const int64_t rows = (int64_t)B * Nm;
-    merge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    launch_dep(merge_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, static_cast<cudaStream_t>(stream), 
         p, N, C, nA - r, Nm, r, static_cast<const __nv_bfloat16*>(x), reinterpret_cast<const int32_t*>(base),
         reinterpret_cast<const int32_t*>(base + cs), reinterpret_cast<int32_t*>(base + 2 * cs),
         static_cast<__nv_bfloat16*>(x_merged), rows);
@@ -858,11 +871,11 @@ extern "C" int usv_unmerge_map(int B, int N, int Nm, const int32_t* pos, int32_t
     cudaError_t e = cudaMemsetAsync(cnt, 0, (size_t)B * Nm * 4, s);
     if (e != cudaSuccess) return fail(USV_ERR_CUDA, "unmerge_map: memset: %s", cudaGetErrorString(e));
     dim3 tg(ceil_div(N, 256), B);
-    inv_count_kernel<<<tg, 256, 0, s>>>(N, Nm, pos, cnt);
+    launch_dep(inv_count_kernel, dim3(tg), dim3(256), 0, s, N, Nm, pos, cnt);
     USV_CHECK_LAUNCH("inv_count_kernel");
-    csr_scan_kernel<<<dim3(ceil_div(Nm, 1024), B), 1024, 0, s>>>(Nm, cnt, inv_off, cursor);
+    launch_dep(csr_scan_kernel, dim3(dim3(ceil_div(Nm, 1024), B)), dim3(1024), 0, s, Nm, cnt, inv_off, cursor);
     USV_CHECK_LAUNCH("csr_scan_kernel");
-    inv_fill_kernel<<<tg, 256, 0, s>>>(N, Nm, pos, cursor, inv_idx);
+    launch_dep(inv_fill_kernel, dim3(tg), dim3(256), 0, s, N, Nm, pos, cursor, inv_idx);
     USV_CHECK_LAUNCH("inv_fill_kernel");
     return USV_OK;
 }

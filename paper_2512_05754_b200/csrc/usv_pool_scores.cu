@@ -31,6 +31,7 @@ constexpr int POOL_SPAN = 4;
 
 template <int D>
 __global__ void __launch_bounds__(128) pool_kernel(const PoolArgs a) {
+    dep_sync();
     constexpr int TPR = D / 8;          // 16 (d=128) or 8 (d=64)
     constexpr int RPI = 128 / TPR;      // rows per iteration: 8 or 16
     constexpr int ITERS = USV_BLOCK / RPI;
@@ -114,6 +115,7 @@ __global__ void __launch_bounds__(256) scores_kernel(const float* __restrict__ q
                                                      const float* __restrict__ kbar,
                                                      float* __restrict__ scores, int NBq, int NBk,
                                                      int d, float scale) {
+    dep_sync();
     constexpr int TM = 64, TN = 64, TK = 32;
     __shared__ __align__(16) float As[TK][TM + 4];
     __shared__ __align__(16) float Bs[TK][TN + 4];
@@ -213,15 +215,15 @@ extern "C" int usv_block_scores(int B, int H, int Nq, int Nk, int d, const void*
     void* tc_mem = reinterpret_cast<char*>(kbar) + align_up((size_t)B * H * NBk * d * sizeof(float), 256);
     if (d == 128) scores_tc_planes(tc_mem, B * H, NBq, NBk, &a.planes[0], &a.planes[1], &a.NB_pad[0], &a.NB_pad[1]);
     dim3 pg(ceil_div(NBq > NBk ? NBq : NBk, POOL_SPAN), B * H, 2);
-    if (d == 128) pool_kernel<128><<<pg, 128, 0, st>>>(a);
-    else pool_kernel<64><<<pg, 128, 0, st>>>(a);
+    if (d == 128) launch_dep(pool_kernel<128>, dim3(pg), dim3(128), 0, st, a);
+    else launch_dep(pool_kernel<64>, dim3(pg), dim3(128), 0, st, a);
     USV_CHECK_LAUNCH("pool_kernel");
 
     if (d == 128)
         return launch_scores_tc(scores, B * H, NBq, NBk, 1.0f / sqrtf((float)d), tc_mem,
                                 static_cast<unsigned int*>(ws), st);
     dim3 sg(ceil_div(NBk, 64), ceil_div(NBq, 64), B * H);
-    scores_kernel<<<sg, 256, 0, st>>>(qbar, kbar, scores, NBq, NBk, d, 1.0f / sqrtf((float)d));
+    launch_dep(scores_kernel, dim3(sg), dim3(256), 0, st, qbar, kbar, scores, NBq, NBk, d, 1.0f / sqrtf((float)d));
     USV_CHECK_LAUNCH("scores_kernel");
     return USV_OK;
 }

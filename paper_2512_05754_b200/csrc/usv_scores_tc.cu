@@ -54,6 +54,7 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 
 __global__ void __launch_bounds__(192, 1)
 scores_tc_kernel(const Args m, const __grid_constant__ Maps maps) {
+    dep_sync();
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -267,7 +268,7 @@ int launch_scores_tc(float* scores, int BH, int NBq, int NBk, float scale, void*
     nz = nz < 1 ? 1 : (nz > t_all ? t_all : nz);
     nz = (t_all + (t_all + nz - 1) / nz - 1) / ((t_all + nz - 1) / nz);   // slices that hold at least one tile
     dim3 grid(m.NBq_pad / 128, BH, nz);
-    sc::scores_tc_kernel<<<grid, 192, sc::SMEM_BYTES, st>>>(m, maps);
+    launch_dep(sc::scores_tc_kernel, dim3(grid), dim3(192), sc::SMEM_BYTES, st, m, maps);
     USV_CHECK_LAUNCH("scores_tc_kernel");
     return USV_OK;
 }

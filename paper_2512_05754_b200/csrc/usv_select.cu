@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* __rest
                                                              int32_t* __restrict__ sel, int H,
                                                              int NBq, int NBk, int kmax,
                                                              const SelHeads heads) {
+    dep_sync();
     extern __shared__ uint32_t keys[];   // NBk order-preserving keys
     __shared__ int hist[256];
     __shared__ int scratch[9];
@@ -155,6 +156,7 @@ __global__ void __launch_bounds__(256, 2) select_warp_kernel(const float* __rest
                                                           int32_t* __restrict__ sel, int H, int NBq,
                                                           int NBk, int kmax, const SelHeads heads,
                                                           int64_t rows) {
+    dep_sync();
     const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (row >= rows) return;
     const int lane = threadIdx.x & 31;
@@ -248,13 +250,13 @@ extern "C" int usv_select_blocks(int B, int H, int NBq, int NBk, const float* sc
     if (rows > 2147483647LL) return fail(USV_ERR_UNSUPPORTED, "select_blocks: too many rows");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const unsigned wg = (unsigned)((rows + 7) / 8);
-#define USV_SEL_WARP(KPL) select_warp_kernel<KPL><<<wg, 256, 0, st>>>(scores, sel, H, NBq, NBk, kmax, heads, rows)
+#define USV_SEL_WARP(KPL) launch_dep(select_warp_kernel<KPL>, dim3(wg), dim3(256), 0, st, scores, sel, H, NBq, NBk, kmax, heads, rows)
     if (NBk <= 256) USV_SEL_WARP(8);
     else if (NBk <= 512) USV_SEL_WARP(16);
     else if (NBk <= 1024) USV_SEL_WARP(32);
     else if (NBk <= 1536) USV_SEL_WARP(48);
     else if (NBk <= 2048) USV_SEL_WARP(64);
-    else select_kernel<<<(unsigned)rows, SEL_THREADS, (size_t)NBk * sizeof(uint32_t), st>>>(scores, sel, H, NBq, NBk, kmax, heads);
+    else launch_dep(select_kernel, dim3((unsigned)rows), dim3(SEL_THREADS), (size_t)NBk * sizeof(uint32_t), st, scores, sel, H, NBq, NBk, kmax, heads);
 #undef USV_SEL_WARP
     USV_CHECK_LAUNCH("select_kernel");
     return USV_OK;
