@@ -135,7 +135,7 @@ __device__ __forceinline__ const int* item_list(const int* hdr) {
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
-    dep_sync();
+    dep_launch();   // the set-up below touches shared and tensor memory only; dep_wait() follows it
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -175,6 +175,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ Maps maps) {
     fence_before();
     __syncthreads();
     fence_after();
+    dep_wait();
     const uint32_t tmem = *s_tmem;
     // Each role starts by handing registers over (service and output warps) or taking them
     // (softmax warps): setmaxnreg, whole warpgroups.
