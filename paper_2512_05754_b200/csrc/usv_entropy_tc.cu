@@ -52,7 +52,7 @@ struct Maps {
 
 __global__ void __launch_bounds__(NTHREADS, 2)
 marginal_tc_kernel(const MargArgs a, const __grid_constant__ Maps maps) {
-    dep_sync();
+    dep_launch();   // the set-up below touches shared and tensor memory only; dep_wait() follows it
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -84,6 +84,7 @@ marginal_tc_kernel(const MargArgs a, const __grid_constant__ Maps maps) {
     fence_before();
     __syncthreads();
     fence_after();
+    dep_wait();
     const uint32_t tmem = *s_tmem;
 
     if (warp == W_TMA) {

@@ -54,7 +54,7 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 
 __global__ void __launch_bounds__(192, 1)
 scores_tc_kernel(const Args m, const __grid_constant__ Maps maps) {
-    dep_sync();
+    dep_launch();   // the set-up below touches shared and tensor memory only; dep_wait() follows it
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -93,6 +93,7 @@ scores_tc_kernel(const Args m, const __grid_constant__ Maps maps) {
     fence_before();
     __syncthreads();
     fence_after();
+    dep_wait();
     const uint32_t tmem = *s_tmem;
 
     if (warp == 4) {
