@@ -87,9 +87,8 @@ static int sparse_attn_impl(int B, int H, int N, int d, const void* q, const usv
     const float sc = scale == 0.f ? 1.0f / sqrtf((float)d) : scale;
     a.scale_log2 = sc * 1.4426950408889634f;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the status word (word 0) is sticky; everything behind it starts at zero
-    cudaError_t e = cudaMemsetAsync(static_cast<char*>(ws) + 4, 0, WS_HEADER - 4, st);
-    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: memset: %s", cudaGetErrorString(e));
+    // the status word (word 0) is sticky; everything behind it starts at zero (the pairing-plan
+    // kernel does that itself: a memset between two kernels costs them their overlapped launch)
     if (impl == 0 && attn_pair_supported(a, d)) {
         int rc2 = launch_pair_plan(a, plan_mem, st);
         if (rc2 != USV_OK) return rc2;
@@ -103,6 +102,8 @@ static int sparse_attn_impl(int B, int H, int N, int d, const void* q, const usv
         return launch_scatter_fallbacks(a, d, st);
     }
     if (y != nullptr) return fail(USV_ERR_UNSUPPORTED, "sparse_attn_unmerge: sequence too long for the tcgen05 kernel");
+    cudaError_t e = cudaMemsetAsync(static_cast<char*>(ws) + 4, 0, WS_HEADER - 4, st);
+    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "sparse_attn: memset: %s", cudaGetErrorString(e));
     return launch_attn_mma(a, d, st);
 }
 

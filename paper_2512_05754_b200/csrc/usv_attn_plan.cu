@@ -31,6 +31,8 @@ constexpr int OVP = CH + 8;     // row pitch of the overlap matrix (uint16): row
 __global__ void __launch_bounds__(THREADS)
 pair_plan_kernel(const AttnArgs a, int2* __restrict__ pairs, int* __restrict__ lists) {
     dep_sync();
+    // the words behind the sticky status word (fallback count, work counter, ...) start at zero
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < (WS_HEADER - 4) / 4) a.status[1 + threadIdx.x] = 0u;
     extern __shared__ __align__(16) uint32_t smem_u[];
     __shared__ int16_t partner[CH];
     __shared__ int16_t best[CH];

@@ -32,6 +32,7 @@ struct MatchTcArgs {
     int* cand_i;                     // [B][nA][2][4] their destination ordinals
     int* exact_list;                 // sources (b * nA + rank) that need the fp32 scan of all destinations
     int* exact_count;
+    int zero_words;              // 32-bit words from exact_count on that half_kernel sets to zero
     unsigned long long* exact_best;  // one slot per list entry: (key of the best cosine << 32) | ~destination
     float* floor_v;                  // [B][nA_pad] lower bound on each source's approximate row maximum
     int32_t* jstar_s;                // [B][nA] best destination TOKEN per source rank

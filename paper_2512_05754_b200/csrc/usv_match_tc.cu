@@ -60,6 +60,8 @@ static_assert(TD + NBUF * 128 <= TMEM_COLS, "TMEM budget");
 __global__ void __launch_bounds__(256)
 half_kernel(const float* __restrict__ mhat, MatchTcArgs m) {
     dep_sync();
+    for (int64_t w = (int64_t)blockIdx.x * 256 + threadIdx.x; w < m.zero_words; w += (int64_t)gridDim.x * 256)
+        reinterpret_cast<unsigned int*>(m.exact_count)[w] = 0u;
     // one warp per output row (4 floats per lane)
     const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
@@ -501,9 +503,10 @@ int launch_match_tc(const float* mhat, const Part& p, int B, int N, int nA, cons
     m.exact_count = reinterpret_cast<int*>(after_list);
     m.exact_best = reinterpret_cast<unsigned long long*>(after_list + 256);
     m.floor_v = reinterpret_cast<float*>(after_list + 256 + 2 * list_bytes(B, N));
-    // counter and result slots of the exact scan start at zero (one memset: they are adjacent)
-    cudaError_t e = cudaMemsetAsync(m.exact_count, 0, 256 + 2 * list_bytes(B, N), st);
-    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: memset: %s", cudaGetErrorString(e));
+    // counter and result slots of the exact scan start at zero: they are adjacent, and half_kernel
+    // clears them (a memset between two kernels costs them their overlapped launch)
+    m.zero_words = (int)((256 + 2 * list_bytes(B, N)) / 4);
+    cudaError_t e;
     const int64_t rows = (int64_t)B * (m.nA_pad + m.nB_pad);
     launch_dep(mt::half_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, st, mhat, m);
     USV_CHECK_LAUNCH("half_kernel");

@@ -264,7 +264,8 @@ __global__ void __launch_bounds__(1024) plan_assign_kernel(Part p, int N, int nA
                                                            int32_t* __restrict__ dst_of,
                                                            int32_t* __restrict__ pos,
                                                            float* __restrict__ u_out,
-                                                           int32_t* __restrict__ jstar_out) {
+                                                           int32_t* __restrict__ jstar_out,
+                                                           int32_t* __restrict__ cnt) {
     dep_sync();
     __shared__ int scratch[33];
     const int b = blockIdx.y;
@@ -320,6 +321,7 @@ __global__ void __launch_bounds__(1024) plan_assign_kernel(Part p, int N, int nA
         const int n = p.dst_token(o);
         d_of[n] = -1;
         ps[n] = nU + o;
+        cnt[(int64_t)b * p.nB + o] = 0;   // the per-destination counts of the CSR pass that follows start at zero
         if (u_out) u_out[(int64_t)b * N + n] = __int_as_float(0x7fc00000);
         if (jstar_out) jstar_out[(int64_t)b * N + n] = -1;
     }
@@ -726,11 +728,12 @@ static int token_merge_impl(int B, int N, int C, const void* x, int Hm, int dm,
         // r = nA: every key is above 0; r = 0: no key is above or equal to the largest one
         dim3 pg(ceil_div(nA > p.nB ? nA : p.nB, 1024), B);
         launch_dep(plan_assign_kernel, dim3(pg), dim3(1024), 0, s, p, N, nA, r, r == nA ? 0u : 0xffffffffu, 0, tsel, src_idx, jstar_s, u_s,
-                                               dst_of, pos, u_out, jstar_out);
+                                               dst_of, pos, u_out, jstar_out, cnt);
         USV_CHECK_LAUNCH("plan_assign_kernel");
+    } else {
+        cudaError_t e = cudaMemsetAsync(cnt, 0, (size_t)B * p.nB * 4, s);
+        if (e != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: memset: %s", cudaGetErrorString(e));
     }
-    cudaError_t e = cudaMemsetAsync(cnt, 0, (size_t)B * p.nB * 4, s);
-    if (e != cudaSuccess) return fail(USV_ERR_CUDA, "token_merge: memset: %s", cudaGetErrorString(e));
     dim3 tg(ceil_div(N, 256), B);
     launch_dep(csr_count_kernel, dim3(tg), dim3(256), 0, s, p, N, nU, dst_of, pos, cnt, row_src);
     USV_CHECK_LAUNCH("csr_count_kernel");
